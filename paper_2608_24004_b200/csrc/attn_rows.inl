@@ -1,6 +1,6 @@
-// Verify attention with the query rows on M, for wide tiles at head_dim 64 (33 .. 128 rows per KV head).
-// Included by attn_tc.cu after its PTX helpers; shares the planner's work items, the tensor maps, the merge
-// kernel and the status word with the keys-on-M kernel there.
+// Verify attention with the query rows on M, for head_dim 64 (up to 256 rows per KV head, in blocks of 128).
+// Included by attn_tc.cu after its PTX helpers; shares the planner's work items, the merge kernel and the status
+// word with the keys-on-M kernel there.
 //
 // Why a second orientation.  With the keys on M a softmax thread owns one key and the rows of a tile are spread
 // over warpgroups, which have to agree on every row's reference (a vote and a rendezvous per tile) and, beyond
@@ -9,45 +9,62 @@
 //     S [128 rows x 128 keys] = Q [128 x D] . K_tile^T          (A = Q, B = K tile, both K-major)
 //     O [128 rows x D]       += P [128 x 128 keys] . V_tile      (A = P from TMEM, written there by the row's own thread; B = V tile, MN-major)
 // a softmax thread owns one query row (one TMEM lane): its running maximum, its row sum, its rescaling of O are
-// its own business, nothing is voted on and nothing is reduced across threads, and one warpgroup of 128 threads
-// does the whole tile at the rate of the transcendental unit (128 x 128 ex2 per tile).  Rows beyond the item's
-// own count are computed and thrown away, so the cost of a tile does not depend on the row count: this form
-// pays off from about 48 rows upward.
+// its own business, nothing is voted on and nothing is reduced across threads.  Rows beyond the item's own count
+// are computed and thrown away, so the cost of a tile depends on the row count only through the number of warps
+// (blocks of 32 rows) that have rows at all.
 //
-// One warpgroup alone leaves the transcendental unit idle most of the time (one warp per scheduler hides no
-// latency, and a tile's softmax is a serial chain of waits, loads, math and arrivals), so the tiles of an item
-// are dealt to NS = 2 independent streams: warpgroup s takes the tiles whose running number is s modulo 2, with
-// its own reference and row sum per row, its own S and P buffer and its OWN accumulator O_s in TMEM.  The two
-// warps that share a scheduler are then half a tile out of phase instead of queueing for the transcendental unit
-// together.  The streams never talk to each other during an item; the epilogue merges the (m, l, O_s) triples of
-// a row like split-KV partials.
+// A tile's softmax is a serial chain (scores out of tensor memory, maximum, 128 exponentials, weights back in), and
+// one warp per scheduler hides none of its latencies, so the tiles of an item are dealt to NS = 2 independent
+// streams: warpgroup s takes the tiles whose running number is s modulo 2, with its own reference and row sum per
+// row, its own S and P buffer and its OWN accumulator O_s in TMEM.  The streams never talk to each other during an
+// item; the epilogue merges the (m, l, O_s) triples of a row like split-KV partials.
 //
-// Warp roles (64 + 128 * NS threads, one CTA per SM, persistent): warp 0 TMA producer (the ring of fused K+V
-// tiles), warp 1 allocates TMEM and one lane issues every tcgen05.mma, then NS softmax warpgroups (lane = row).
+// Softmax of a tile, per thread: pass 1 takes the row maximum of the 128 scores; the row's reference follows it
+// lazily (it moves, and O_s and the row sum are rescaled, only when the maximum exceeds it by more than 2^8); pass 2
+// turns the scores into weights 2^(score - reference).  The scores have left tensor memory for good a quarter of
+// the way before the end of pass 2; from then on the stream's S buffer is free (s_free) and the QK product of the
+// stream's next tile runs under the rest of this tile's weights.
+//
+// K and V tiles travel in separate rings (3 + 8 slots of 16 KB), each filled by its own producer warp: a K tile is
+// dead as soon as its QK product has completed, a V tile has to wait for the whole softmax of its tile, and in one
+// ring of fused K+V slots the K halves would hold their shared memory for all that time; the depth of the prefetch,
+// not the arithmetic, bounded the kernel then (five fused slots: 1590 cycles a tile, four: 1820).
+//
+// Warps (352 threads, one CTA per SM, persistent): 0..7 softmax (stream = warp / 4, TMEM lane quarter = warp % 4),
+// 8 K producer, 9 V producer, 10 issues every tcgen05.mma from one lane.  Issuing a product costs that lane 50 cycles
+// when it has its scheduler to itself and up to twice that when softmax warps compete for the issue slots; at twelve
+// products a tile it is what bounds wide tiles.  A warp's scheduler is its index modulo 4, and so is its TMEM lane
+// quarter: warp 10 shares scheduler 2 with the softmax warps of lanes 64..95, and the block's rows 96..127, the ones
+// that most items do not have, are mapped to those lanes (rows 64..95 to lanes 96..127).
 // Every wait is bounded as in the other kernel.
 
 template <int D, int NS>
 struct RowsSmem {
   static_assert(D == 64, "rows-on-M kernel: head_dim 64");
   static constexpr int kRows = 128;
-  static constexpr int kSlotBytes = kTile * D * 2 * 2;         // fused K + V tile
+  static constexpr int kTileBytes = kTile * D * 2;             // one K or V tile
   static constexpr int kQBytes = kRows * D * 2;
   static constexpr int kPBufs = 2;                             // P buffers, in TMEM
   static constexpr int kMlBytes = 2 * NS * kRows * 8;          // per item parity, stream and row: (m, l)
   static constexpr int kSmallBytes = 40 * 8 + 256 + kMlBytes + kItemCache * 32;
   static constexpr int kQBufs = 2;                             // the next item's queries are staged during this one
   static constexpr int kFree = 232448 - 1024 - kQBufs * kQBytes - kSmallBytes;
-  static constexpr int kSlots = kFree / kSlotBytes > 8 ? 8 : kFree / kSlotBytes;
-  static_assert(kSlots >= 3, "the K/V ring needs at least three slots");
-  static constexpr int kOffQ = kSlots * kSlotBytes;
+  static constexpr int kKSlots = 3;
+  static constexpr int kVSlots = kFree / kTileBytes - kKSlots > 8 ? 8 : kFree / kTileBytes - kKSlots;
+  static_assert(kKSlots >= 2 && kVSlots >= 3, "rings too shallow");
+  static_assert((kKSlots + kVSlots) * kTileBytes <= kFree, "rings do not fit");
+  static constexpr int kOffK = 0;
+  static constexpr int kOffV = kKSlots * kTileBytes;
+  static constexpr int kOffQ = (kKSlots + kVSlots) * kTileBytes;
   static constexpr int kOffBars = kOffQ + kQBufs * kQBytes;
-  static constexpr int kNumBars = 2 * kSlots + 15;
+  static constexpr int kNumBars = 2 * (kKSlots + kVSlots) + 15;
   static_assert(kNumBars <= 40, "barrier reservation");
   static constexpr int kOffCtl = kOffBars + 40 * 8;
   static constexpr int kOffMl = kOffCtl + 256;
   static constexpr int kOffItems = kOffMl + kMlBytes;
   static constexpr int kTotal = kOffItems + kItemCache * 32;
-  static constexpr int kThreads = 64 + 128 * NS;
+  static constexpr int kWarpProdK = 4 * NS, kWarpProdV = 4 * NS + 1, kWarpMma = 4 * NS + 2, kWarps = 4 * NS + 3;
+  static constexpr int kThreads = 32 * kWarps;
   // TMEM columns: S0, S1 (128 each), O_0 .. O_{NS-1} (D each), P0, P1 (64 each: 128 bf16 weights per row, two to a column)
   static constexpr uint32_t kTmemCols = 512;
   static_assert(2 * kTile + NS * D + kPBufs * (kTile / 2) <= 512, "S, O and P must fit in TMEM");
@@ -70,7 +87,12 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
 }
-constexpr float kRescaleSum = 512.f;             // a tile's weights of one row may add up to this before its reference moves
+constexpr float kRescaleStep = 8.f;              // a row's reference moves when a tile's maximum exceeds it by more than this (log2 units)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 
 // tcgen05.mma with the A operand in tensor memory (row = lane, two bf16 per 32-bit column)
 __device__ __forceinline__ void umma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
@@ -106,35 +128,160 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* r) {
       : "memory");
 }
 
+// Non-blocking look at four mbarriers: bit i = phase `parity i` of barrier i is complete.
+__device__ __forceinline__ uint32_t mbar_test4(uint32_t bar0, uint32_t par0, uint32_t bar1, uint32_t par1, uint32_t bar2,
+                                               uint32_t par2, uint32_t bar3, uint32_t par3) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p0, p1, p2, p3;\n\t.reg .u32 a, b, c, d;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p0, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p1, [%3], %4;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p2, [%5], %6;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p3, [%7], %8;\n\t"
+      "selp.u32 a, 1, 0, p0;\n\t"
+      "selp.u32 b, 2, 0, p1;\n\t"
+      "selp.u32 c, 4, 0, p2;\n\t"
+      "selp.u32 d, 8, 0, p3;\n\t"
+      "or.b32 a, a, b;\n\t"
+      "or.b32 c, c, d;\n\t"
+      "or.b32 %0, a, c;\n\t}"
+      : "=r"(r)
+      : "r"(bar0), "r"(par0), "r"(bar1), "r"(par1), "r"(bar2), "r"(par2), "r"(bar3), "r"(par3)
+      : "memory");
+  return r;
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // An item with more than 128 query rows is walked once per block of 128 rows: the same keys again, the next rows.
 // Every role derives the number of blocks from the item itself (G = query heads per kv head).
 __device__ __forceinline__ int row_blocks_of(int G, const ItemView& v) { return (G * (v.k + 1) + 127) / 128; }
 
+constexpr float kGrowSum = 512.f;                // a tile's weights of one row may add up to this before its reference moves
+constexpr float kHugeSum = 7.9e28f;              // 2^96: beyond it (or NaN) the weights may have overflowed
+
+// The softmax of one tile for one warp's rows WITHOUT the scores in tensor memory: every thread recomputes its row's
+// 128 scores from the queries and keys in global memory (fp32 sums of the exact bf16 products), takes their maximum as
+// the row's new reference, rescales its row of O_s and its sum, and writes the weights.  Slow (two passes of 128 dot
+// products per thread) and rare: the optimistic pass of the kernel calls it when a row's weights overflowed, which
+// takes a score more than 2^96 above the row's reference, long after the scores were released.  All 32 lanes call it.
+template <int D>
+__device__ __noinline__ void rows_tile_from_memory(const __nv_bfloat16* qrow, const __nv_bfloat16* k_pool, const int32_t* bt_row,
+                                                   int bs, int Hkv, int head, int num_blocks, int kbase, int key_end, int hi_r,
+                                                   int lo_r, float scale, uint32_t p_addr, uint32_t os_addr, bool own_first, float& m,
+                                                   float& l) {
+  float q[D];
+  if (qrow) {
+#pragma unroll
+    for (int x = 0; x < D / 8; ++x) {
+      const uint4 u = __ldg(reinterpret_cast<const uint4*>(qrow) + x);
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        q[8 * x + 2 * y] = __uint_as_float(w[y] << 16);
+        q[8 * x + 2 * y + 1] = __uint_as_float(w[y] & 0xffff0000u);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int d = 0; d < D; ++d) q[d] = 0.f;
+  }
+  auto score = [&](int t) -> float {
+    const int tt = kbase + t;
+    if (tt >= key_end || tt > hi_r || tt < lo_r) return -INFINITY;
+    const int page = __ldg(bt_row + tt / bs);
+    if ((unsigned)page >= (unsigned)num_blocks) return -INFINITY;
+    const uint4* kr = reinterpret_cast<const uint4*>(k_pool + ((size_t)(page * Hkv + head) * bs + tt % bs) * D);
+    float acc = 0.f;
+#pragma unroll
+    for (int x = 0; x < D / 8; ++x) {
+      const uint4 u = __ldg(kr + x);
+      const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        acc = fmaf(q[8 * x + 2 * y], __uint_as_float(w[y] << 16), acc);
+        acc = fmaf(q[8 * x + 2 * y + 1], __uint_as_float(w[y] & 0xffff0000u), acc);
+      }
+    }
+    return acc;
+  };
+  float mx = -INFINITY;
+#pragma unroll 1
+  for (int t = 0; t < kTile; ++t) mx = fmaxf(mx, score(t));
+  const float mnew = fmaxf(m, mx * scale);
+  const float alpha = m == -INFINITY ? 0.f : exp2f(m - mnew);
+  if (!own_first) {
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      float o[32];
+      tmem_ld32(os_addr + c * 32, o);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) o[e] *= alpha;
+      tmem_st32(os_addr + c * 32, o);
+    }
+    tmem_wait_st();
+  }
+  l *= alpha;
+  m = mnew;
+  const float mref = m == -INFINITY ? 0.f : m;
+  float lt = 0.f;
+#pragma unroll 1
+  for (int c = 0; c < kTile / 32; ++c) {
+    uint32_t pk[16];
+#pragma unroll 1
+    for (int e = 0; e < 32; e += 2) {
+      const float p0 = exp2f(fmaf(score(c * 32 + e), scale, -mref)), p1 = exp2f(fmaf(score(c * 32 + e + 1), scale, -mref));
+      lt += p0 + p1;
+      const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+      const uint32_t word = *reinterpret_cast<const uint32_t*>(&pb);
+      // (pk is filled through a constant-index switch so that it stays in registers under the rolled loop)
+#pragma unroll
+      for (int x = 0; x < 16; ++x)
+        if (x == (e >> 1)) pk[x] = word;
+    }
+    tmem_st16u(p_addr + c * 16, pk);
+  }
+  tmem_wait_st();
+  l += lt;
+}
+
 template <int D, int NS>
 __global__ void __launch_bounds__(RowsSmem<D, NS>::kThreads, 1)
-attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs A) {
+attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, DevPlan P, AttnArgs A) {
   using L = RowsSmem<D, NS>;
-  constexpr int kSlots = L::kSlots;
+  constexpr int KS = L::kKSlots, VS = L::kVSlots;
   constexpr int kThreads = L::kThreads;
   constexpr int NP = L::kPBufs;
   constexpr int KSTEPS_S = D / 16;
   constexpr int KSTEPS_PV = kTile / 16;
-  constexpr uint32_t SBO_KV = 2048;                     // 8-key group stride inside a fused slot
-  const uint32_t k_off = A.fused_k_first ? 0u : 1024u;
-  const uint32_t v_off = A.fused_k_first ? 1024u : 0u;
+  constexpr uint32_t SBO_KV = 1024;                     // 8-key group stride inside a K or V tile
   constexpr uint32_t TMEM_COLS = L::kTmemCols;
 
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bars = sbase + L::kOffBars;
-  auto bar_slot_full = [&](int s) { return bars + 8u * s; };
-  // completion of the PV product of tile h, on barrier h % kSlots: frees the tile's K/V slot for the producer and
+  auto bar_k_full = [&](int s) { return bars + 8u * s; };
+  // the K slot of tile g is released by the stream that has seen the tile's scores complete
+  auto bar_k_empty = [&](int s) { return bars + 8u * (KS + s); };
+  auto bar_v_full = [&](int s) { return bars + 8u * (2 * KS + s); };
+  // completion of the PV product of tile h, on barrier h % VS: frees the tile's V slot for the producer and
   // its P buffer for the softmax threads, and tells them that O holds the products up to tile h (one commit
-  // instead of two: every commit costs the issuing thread about as much as a product)
-  auto bar_slot_empty = [&](int s) { return bars + 8u * (kSlots + s); };
-  static_assert(kSlots >= NP + 1, "a P buffer is reused before its tile's slot");
-  const uint32_t b0 = bars + 8u * 2 * kSlots;
+  // for all three: every commit costs the issuing thread about as much as a product)
+  auto bar_v_empty = [&](int s) { return bars + 8u * (2 * KS + VS + s); };
+  static_assert(VS >= NP + 1, "a P buffer is reused before its tile's slot");
+  const uint32_t b0 = bars + 8u * 2 * (KS + VS);
   auto bar_s_full = [&](int b) { return b0 + 8u * b; };
   auto bar_s_free = [&](int b) { return b0 + 8u * (2 + b); };
   auto bar_p_full = [&](int b) { return b0 + 8u * (4 + b); };
@@ -150,9 +297,13 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
   const int it_begin = A.cta_first[blockIdx.x], it_end = A.cta_first[blockIdx.x + 1];
 
   if (tid == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(bar_slot_full(s), 1);
-      mbar_init(bar_slot_empty(s), 1);
+    for (int s = 0; s < KS; ++s) {
+      mbar_init(bar_k_full(s), 1);
+      mbar_init(bar_k_empty(s), 1);
+    }
+    for (int s = 0; s < VS; ++s) {
+      mbar_init(bar_v_full(s), 1);
+      mbar_init(bar_v_empty(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_s_full(b), 1);
@@ -175,7 +326,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
   // Q staging starts out as zeros: rows that no item uses stay finite
   for (int x = tid; x < L::kQBufs * L::kQBytes / 16; x += kThreads)
     reinterpret_cast<uint4*>(smem + L::kOffQ)[x] = make_uint4(0, 0, 0, 0);
-  if (warp == 1) {
+  if (warp == L::kWarpMma) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"(TMEM_COLS)
                  : "memory");
@@ -188,74 +339,81 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s0 = tmem, tmem_o = tmem + 2 * kTile, tmem_p0 = tmem_o + NS * D;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer (one fused K+V copy per page)
+  if (warp == L::kWarpProdK || warp == L::kWarpProdV) {
+    // ------------------------------------------------------------------ TMA producers: one ring each, one copy per page
+    const bool is_k = warp == L::kWarpProdK;
+    const CUtensorMap* map = is_k ? &kmap : &vmap;
+    const int NSLOT = is_k ? KS : VS;
+    const uint32_t ring = sbase + (is_k ? L::kOffK : L::kOffV);
     const int pages_per_tile = kTile / P.bs;
-    const uint32_t page_bytes = (uint32_t)P.bs * D * 2 * 2;
-    uint32_t load_idx = 0;
-    bool ok = it_begin < it_end;
-    int it = it_begin, tile = 0;
-    int rb = 0;                                            // row block of the item (see row_blocks_of)
-    ItemView v = ok ? view(A, item_cache, it_begin, it) : ItemView{};
-    auto fetch_page = [&](const ItemView& iv, int tl) -> int {
-      const int kb = iv.key_begin + tl * kTile;
-      const int np = min(pages_per_tile, (iv.key_end - kb + P.bs - 1) / P.bs);
-      return lane < np ? __ldg(A.block_table + (size_t)iv.req * P.max_blocks + kb / P.bs + lane) : -1;
+    const uint32_t page_bytes = (uint32_t)P.bs * D * 2;
+    // Page ids come 32 at a time (one coalesced load of the request's block-table row: four tiles' worth at 16 keys a
+    // page), a chunk ahead of their use: a load per tile, even issued a tile early, put a global-memory round trip
+    // into every pass of this loop and held a producer to one tile per ~1500 cycles.
+    const int tiles_per_chunk = 32 / pages_per_tile;
+    auto chunk_load = [&](const ItemView& v, int c) -> int {
+      const int idx = c * 32 + lane;                       // page of the item's key range
+      const int np_item = (v.key_end - v.key_begin + P.bs - 1) / P.bs;
+      return idx < np_item ? __ldg(A.block_table + (size_t)v.req * P.max_blocks + v.key_begin / P.bs + idx) : -1;
     };
-    int page_raw = ok ? fetch_page(v, 0) : -1;
+    uint32_t load_idx = 0;                                 // running tile number
+    bool ok = it_begin < it_end;
+    int it = it_begin, rb = 0;
+    ItemView v = ok ? view(A, item_cache, it_begin, it_begin) : ItemView{};
+    int ids = ok ? chunk_load(v, 0) : -1;
     while (ok) {
-      int nit = it, nrb = rb, ntile = tile + 1;
+      // the (item, row block) that follows this one: the same keys again for the item's next 128 rows, or the next item
+      int nit = it, nrb = rb + 1;
       ItemView nv = v;
-      if (ntile == v.tiles && rb + 1 < row_blocks_of(G, v)) {     // the same keys again, for the item's next 128 rows
-        nrb = rb + 1;
-        ntile = 0;
-      } else if (ntile == v.tiles) {
-        nit = it + 1;
+      if (nrb == row_blocks_of(G, v)) {
         nrb = 0;
-        ntile = 0;
+        nit = it + 1;
         if (nit < it_end) nv = view(A, item_cache, it_begin, nit);
       }
-      const bool more = nit < it_end;
-      const int next_raw = more ? fetch_page(nv, ntile) : -1;
-      const int kbase = v.key_begin + tile * kTile;
-      const int npages = min(pages_per_tile, (v.key_end - kbase + P.bs - 1) / P.bs);
-      int page = page_raw;
-      if (lane < npages && (unsigned)page >= (unsigned)P.num_blocks) {
-        atomicOr(P.status, kFlagBadPage);
-        page = -1;
+      const int nch = (v.tiles + tiles_per_chunk - 1) / tiles_per_chunk;
+      for (int c = 0; c < nch && ok; ++c) {
+        const int ids_next = c + 1 < nch ? chunk_load(v, c + 1) : (nit < it_end ? chunk_load(nv, 0) : -1);
+        const int t_end = min(v.tiles, (c + 1) * tiles_per_chunk);
+        for (int tile = c * tiles_per_chunk; tile < t_end; ++tile) {
+          const int kbase = v.key_begin + tile * kTile;
+          const int npages = min(pages_per_tile, (v.key_end - kbase + P.bs - 1) / P.bs);
+          int page = __shfl_sync(0xffffffffu, ids, ((tile - c * tiles_per_chunk) * pages_per_tile + lane) & 31);
+          if (lane >= npages) page = -1;
+          if (lane < npages && (unsigned)page >= (unsigned)P.num_blocks) {
+            atomicOr(P.status, kFlagBadPage);
+            page = -1;
+          }
+          const int nvalid = __popc(__ballot_sync(0xffffffffu, page >= 0));
+          const int slot = load_idx % NSLOT;
+          const uint32_t par = ((load_idx / NSLOT) & 1u) ^ 1u;
+          const uint32_t full = is_k ? bar_k_full(slot) : bar_v_full(slot);
+          int good = 1;
+          if (lane == 0) good = mbar_wait_c(is_k ? bar_k_empty(slot) : bar_v_empty(slot), par, ctl, P.status, is_k ? 0 : 1) ? 1 : 0;
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
+          if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)nvalid * page_bytes);
+          __syncwarp();
+          if (page >= 0)
+            tma_load_5d(ring + slot * L::kTileBytes + lane * page_bytes, map, full, 0, 0, 0, 0, page * P.Hkv + v.kv_head);
+          ++load_idx;
+        }
+        ids = ids_next;
       }
-      const int nvalid = __popc(__ballot_sync(0xffffffffu, page >= 0));
-      const int slot = load_idx % kSlots;
-      const uint32_t par = ((load_idx / kSlots) & 1u) ^ 1u;
-      int good = 1;
-      if (lane == 0) good = mbar_wait_c(bar_slot_empty(slot), par, ctl, P.status, 0) ? 1 : 0;
-      good = __shfl_sync(0xffffffffu, good, 0);
-      if (!good) break;
-      if (lane == 0) mbar_arrive_expect_tx(bar_slot_full(slot), (uint32_t)nvalid * page_bytes);
-      __syncwarp();
-      if (page >= 0)
-        tma_load_5d(sbase + slot * L::kSlotBytes + lane * page_bytes, &kvmap, bar_slot_full(slot), 0, 0, 0, 0,
-                    page * P.Hkv + v.kv_head);
-      ++load_idx;
-      if (!more) break;
+      if (nit >= it_end) break;
       it = nit;
       rb = nrb;
-      tile = ntile;
       v = nv;
-      page_raw = next_raw;
     }
-  } else if (warp == 1) {
+  } else if (warp == L::kWarpMma) {
     // ------------------------------------------------------------------ MMA issuer (one lane)
     if (lane == 0) {
       constexpr uint32_t idesc_s = instr_desc(L::kRows, kTile, false, false);   // S: M = 128 rows, N = 128 keys
       constexpr uint32_t idesc_pv = instr_desc(L::kRows, D, false, true);       // O: M = 128 rows, N = head_dim, B = V MN-major
-      // Two cursors over this CTA's tiles.  Every operation of this thread that touches the tensor unit or a
-      // barrier costs it 60-140 cycles (a product about 75, a commit about 130, a look at the barriers about
-      // 140, a fence 60), and at twelve products a tile that thread is what bounds the kernel; so a pass of the
-      // loop below does as much as possible on one look and one fence.  In the steady state the arrival of a
-      // stream's weights P(h) triggers one pass: the QK product of that stream's NEXT tile h + 2 first (its S
-      // buffer is free, because the stream arrives on s_free before p_full), then the PV product of tile h.  The
-      // stream is back at work after one short product, and the other stream's tile h + 1 overlaps both.
+      // Two cursors over this CTA's tiles: cs for the QK products, cp for the PV products.  Every operation of this
+      // thread that touches the tensor unit or a barrier costs it 50-140 cycles, so a pass of the loop below looks at
+      // all the barriers it may need at once.  QK(g) needs the tile's K slot and the stream's S buffer (s_free: the
+      // stream has taken the scores of its previous tile out of tensor memory); PV(g) needs the weights P(g) and the
+      // tile's V slot.  Whichever is ready goes, in any order: nothing here can wait for something it has yet to issue.
       struct Cursor {
         int it, rb;
         int tile;
@@ -278,26 +436,21 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
       unsigned long long idle_since = 0;
       uint32_t spins = 0;
       while (cp.it < it_end) {
-        const bool s_cand = cs.it < it_end && cs.g <= cp.g + 2;
+        const bool s_cand = cs.it < it_end;
         const bool p_cand = cp.g < cs.g;
-        const int kslot = cs.g % kSlots, sbuf = cs.g & 1;
-        const int vslot = cp.g % kSlots, pbuf = cp.g % NP;
-        // one look: the K/V slot of the next QK product, its S buffer, the weights of the next PV product
-        const uint32_t rdy = mbar_test3(bar_slot_full(kslot), (cs.g / kSlots) & 1u, bar_s_free(sbuf), ((cs.g >> 1) & 1u) ^ 1u,
-                                        bar_p_full(pbuf), (cp.g / NP) & 1u);
+        const int kslot = cs.g % KS, sbuf = cs.g & 1;
+        const int vslot = cp.g % VS, pbuf = cp.g % NP;
+        const uint32_t rdy = mbar_test4(bar_k_full(kslot), (cs.g / KS) & 1u, bar_s_free(sbuf), ((cs.g >> 1) & 1u) ^ 1u,
+                                        bar_p_full(pbuf), (cp.g / NP) & 1u, bar_v_full(vslot), (cp.g / VS) & 1u);
         const bool p_first = cp.tile < NS;                 // the first tile of its stream in this item
-        bool p_ok = p_cand && (rdy & 4u);
-        if (p_ok && p_first) p_ok = mbar_test3(bar_o_free, (cp.item_idx & 1u) ^ 1u, bar_o_free, (cp.item_idx & 1u) ^ 1u, bar_o_free,
-                                               (cp.item_idx & 1u) ^ 1u) == 7u;   // the last item's O has been read
-        // (two tiles ahead the S buffer is the one whose weights the PV product of this pass consumes)
-        bool s_ok = s_cand && (rdy & 1u) && (cs.g == cp.g + 2 ? p_ok : (rdy & 2u) != 0);
-        if (s_ok && cs.tile == 0)
-          s_ok = mbar_test3(bar_q_full(cs.item_idx & 1u), (cs.item_idx >> 1) & 1u, bar_q_full(cs.item_idx & 1u), (cs.item_idx >> 1) & 1u,
-                            bar_q_full(cs.item_idx & 1u), (cs.item_idx >> 1) & 1u) == 7u;
+        bool p_ok = p_cand && (rdy & 12u) == 12u;
+        if (p_ok && p_first) p_ok = mbar_test(bar_o_free, (cp.item_idx & 1u) ^ 1u);   // the last item's O has been read
+        bool s_ok = s_cand && (rdy & 3u) == 3u;
+        if (s_ok && cs.tile == 0) s_ok = mbar_test(bar_q_full(cs.item_idx & 1u), (cs.item_idx >> 1) & 1u);
         if (s_ok || p_ok) tc_fence_after();
         if (s_ok) {
           // A = Q, B = K tile (both K-major, 128-byte swizzle): 32 bytes per step inside the 64-element atom
-          const uint32_t k_lo = desc_lo(sbase + kslot * L::kSlotBytes + k_off, 16);
+          const uint32_t k_lo = desc_lo(sbase + L::kOffK + kslot * L::kTileBytes, 16);
           const uint32_t q_lo = desc_lo(sbase + L::kOffQ + (cs.item_idx & 1u) * L::kQBytes, 16);
 #pragma unroll
           for (int kk = 0; kk < KSTEPS_S; ++kk)
@@ -311,12 +464,12 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
           // A = P from TMEM (row = lane, 16 keys of a step = 8 columns); B = V (MN-major, 128-byte swizzle):
           // 16 keys per step = two 8-key groups
           const uint32_t p_t = tmem_p0 + pbuf * (kTile / 2);
-          const uint32_t v_lo = desc_lo(sbase + vslot * L::kSlotBytes + v_off, 1024);
+          const uint32_t v_lo = desc_lo(sbase + L::kOffV + vslot * L::kTileBytes, 1024);
 #pragma unroll
           for (int kk = 0; kk < KSTEPS_PV; ++kk)          // tile g belongs to stream g % NS and accumulates into its O
             umma_bf16_ta(tmem_o + (cp.g % NS) * D, p_t + kk * 8, v_lo + kk * (2 * SBO_KV / 16), desc_hi(SBO_KV, 2), idesc_pv,
                          !(p_first && kk == 0));
-          umma_commit(bar_slot_empty(vslot));
+          umma_commit(bar_v_empty(vslot));
           if (cp.tile == cp.v.tiles - 1) umma_commit(bar_o_full);
           advance(cp);
         }
@@ -339,9 +492,12 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue (thread = query row)
-    const int stream = (warp - 2) >> 2;                   // which tiles: those whose running number is `stream` modulo NS
-    const int quarter = warp & 3;                         // TMEM lanes this warp may touch
-    const int r = quarter * 32 + lane;                    // query row of the tile = TMEM lane
+    const int stream = warp >> 2;                         // which tiles: those whose running number is `stream` modulo NS
+    const int quarter = warp & 3;                         // TMEM lanes this warp may touch: 32 * quarter ..
+    const int rp = quarter * 32 + lane;                   // this thread's TMEM lane = row of the Q operand
+    // ... and which 32 rows of a block live there: rows 96..127 on the lanes of the issuing warp's scheduler
+    const int lq = quarter == 2 ? 3 : (quarter == 3 ? 2 : quarter);
+    const int r = lq * 32 + lane;                         // this thread's query row of the block
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     constexpr int CK = kTile;
     constexpr int NCH = CK / 32;                          // a tile's keys in chunks of 32
@@ -367,19 +523,19 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
       const int qb = item_idx & 1u;
       if (!mbar_wait_c(bar_q_free(qb), ((item_idx >> 1) & 1u) ^ 1u, ctl, P.status, 8)) return false;
       constexpr int CPT = D / 8 / NS;
-      const uint32_t qrow = sbase + L::kOffQ + qb * L::kQBytes + r * 128;
+      const uint32_t qrow = sbase + L::kOffQ + qb * L::kQBytes + rp * 128;
       const int j = rb * L::kRows + r;                      // row of the item
       if (j < G * (v.k + 1)) {
         const __nv_bfloat16* src = A.q + ((size_t)(v.cu_q + j / G) * P.Hq + v.kv_head * G + j % G) * D;
 #pragma unroll
         for (int x = 0; x < CPT; ++x)
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(qrow + (((stream * CPT + x) ^ (r & 7)) << 4)),
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(qrow + (((stream * CPT + x) ^ (rp & 7)) << 4)),
                        "l"(src + (stream * CPT + x) * 8)
                        : "memory");
       } else {
 #pragma unroll
         for (int x = 0; x < CPT; ++x)
-          *reinterpret_cast<uint4*>(smem + L::kOffQ + qb * L::kQBytes + r * 128 + (((stream * CPT + x) ^ (r & 7)) << 4)) =
+          *reinterpret_cast<uint4*>(smem + L::kOffQ + qb * L::kQBytes + rp * 128 + (((stream * CPT + x) ^ (rp & 7)) << 4)) =
               make_uint4(0, 0, 0, 0);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
@@ -402,12 +558,14 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
       if (rb == row_blocks_of(G, v)) break;
       const int R = G * (v.k + 1) - rb * L::kRows;        // rows of the item from this block's first on
       const int j = rb * L::kRows + r;                    // this thread's row of the item
-      const bool warp_active = quarter * 32 < R;          // some row of this warp belongs to the item
+      const bool warp_active = lq * 32 < R;               // some row of this warp belongs to the item
       // keys this row may see: lo_r .. hi_r.  A row beyond the item's own (its queries are zeros) sees everything:
       // it costs its warp no masking, and what it computes is never stored.
       const int hi_r = r < R ? v.n + j / G : 0x7fffffff;
       const int lo_r = (r < R && W > 0) ? max(0, hi_r - W + 1) : 0;
       float m = -INFINITY, l = 0.f;                       // this stream's running reference (log2 units) and row sum
+      float o_alpha = 1.f;                                // factor this row of O_s is still owed (see the optimistic pass)
+      bool o_owed = false;                                // ... for some row of the warp
       bool own_first = true;                              // the stream has not had a tile of this item yet
       // the queries of the next (item, row block) start their way into the other Q buffer now
       bool q_pending = false;
@@ -424,9 +582,23 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
         const int kbase = v.key_begin + tile * kTile;
         const int sbuf = g & 1, pbuf = g % NP;
         if (!mbar_wait_c(bar_s_full(sbuf), (g >> 1) & 1u, ctl, P.status, 9)) { ok = false; break; }
+        // the tile's scores are complete, so its K slot has served its purpose
+        if (quarter == 0 && lane == 0) mbar_arrive(bar_k_empty(g % KS));
         tc_fence_after();
-        // the P buffer of this tile becomes writable when the PV product that last read it (tile g - NP) is done
-        if (g >= (uint32_t)NP && !mbar_wait_c(bar_slot_empty((g - NP) % kSlots), ((g - NP) / kSlots) & 1u, ctl, P.status, 10)) { ok = false; break; }
+        // the P buffer of this tile becomes writable when the PV product that last read it (tile g - NP) is done: not
+        // needed before the row maxima are known.  (That product is also the last that O_s was waiting for.)
+        static_assert(NP == NS, "the P buffer's last reader is the stream's previous tile");
+        auto wait_p = [&]() -> bool {
+          return g < (uint32_t)NP || mbar_wait_c(bar_v_empty((g - NP) % VS), ((g - NP) / VS) & 1u, ctl, P.status, 10);
+        };
+        // All of a tile's scores have left tensor memory some way before its weights are finished: from then on the
+        // issuing thread may compute the stream's next scores into the same buffer (arrival on s_free).
+        bool s_released = false;
+        auto release_s = [&]() {
+          tc_fence_before();
+          warp_arrive(bar_s_free(sbuf));
+          s_released = true;
+        };
         if (warp_active) {
           const uint32_t s_addr = tmem_s0 + sbuf * kTile + lane_addr;
           const uint32_t p_addr = tmem_p0 + pbuf * (kTile / 2) + lane_addr;
@@ -434,134 +606,229 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
           // every row of the warp sees every key of the tile: the common case, which then
           // carries no masking code at all (a per-thread test is compiled into selects that every tile pays for)
           const bool interior = __all_sync(0xffffffffu, t_first >= lo_r && t_first + CK - 1 <= hi_r);
-          // 32 raw scores of this row, -inf where the row may not see the key
-          auto scores = [&](int c, float* y, auto masked) {
-            tmem_ld32(s_addr + c * 32, y);
-            tmem_wait_ld();
-            if constexpr (decltype(masked)::value) {
-              const int t0 = t_first + c * 32;
+          auto max32 = [&](float mx, const float* y) -> float {      // (four chains: a single one is 16 dependent steps)
+            float a = mx, b = y[0], c = y[1], d = y[2];
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (t0 + e > hi_r || t0 + e < lo_r) y[e] = -INFINITY;
+            for (int e = 3; e + 7 < 32; e += 8) {
+              a = fmax3(a, y[e], y[e + 1]);
+              b = fmax3(b, y[e + 2], y[e + 3]);
+              c = fmax3(c, y[e + 4], y[e + 5]);
+              d = fmax3(d, y[e + 6], y[e + 7]);
+            }
+            // (e = 3, 11, 19 covered y[3..26])
+            a = fmax3(a, y[27], y[28]);
+            b = fmax3(b, y[29], y[30]);
+            c = fmaxf(c, y[31]);
+            return fmax3(fmaxf(a, b), c, d);
+          };
+          // weights 2^(score - reference) of 32 keys in bf16 into the P buffer, their sum into acc.  The subtraction and
+          // the row sum run on packed pairs (fma / add .f32x2).
+          auto chunk_pack = [&](const float* y, uint64_t sc2, uint64_t nm2, uint64_t* acc, uint32_t* pk) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              float d0, d1;
+              unpack2(fma2(pack2(y[e], y[e + 1]), sc2, nm2), d0, d1);
+              const float p0 = exp2f(d0), p1 = exp2f(d1);
+              acc[(e >> 1) & 3] = add2(acc[(e >> 1) & 3], pack2(p0, p1));
+              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
             }
           };
-          // weights 2^(score - reference) of the row's keys in bf16 into the P buffer; returns their sum.  The
-          // subtraction and the row sum run on packed pairs (fma / add .f32x2): the softmax warps are bound by
-          // instruction issue, not by the transcendental unit.
-          auto weights = [&](float mref, auto masked) -> float {
+          auto chunk_weights = [&](int c, const float* y, uint64_t sc2, uint64_t nm2, uint64_t* acc) {
+            uint32_t pk[16];
+            chunk_pack(y, sc2, nm2, acc, pk);
+            tmem_st16u(p_addr + c * 16, pk);              // 32 keys = 16 columns of the row's lane
+          };
+          // The row's reference follows its running maximum lazily: it moves only when the tile's maximum exceeds it by
+          // more than 2^kRescaleStep (weights up to that size are harmless), which after the first tiles is rare.  When
+          // it moves for some row of the warp, the warp rescales its rows of O_s (a collective access) and its sums.
+          // Only the item's own rows vote: a lane beyond them multiplies zero queries with whatever the slot holds.
+          // The P buffer is writable, and O_s holds the products up to the stream's previous tile, once that tile's PV
+          // product is done.
+          bool p_waited = false;
+          if (o_owed || !interior) {
+            if (!wait_p()) { ok = false; break; }
+            p_waited = true;
+          }
+          // factor by which this row of O_s is to be multiplied (collective: every lane of the warp takes part)
+          auto scale_o = [&](float f) {
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              float o[32];
+              tmem_ld32(tmem_os + lane_addr + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] *= f;
+              tmem_st32(tmem_os + lane_addr + c * 32, o);
+            }
+            tmem_wait_st();
+          };
+          if (o_owed) {                                     // a reference moved after the previous tile's weights were out
+            scale_o(o_alpha);
+            o_alpha = 1.f;
+            o_owed = false;
+          }
+          // The row's reference follows its running maximum lazily: it moves only when the tile's maximum exceeds it by
+          // more than 2^kRescaleStep (weights up to that size are harmless).  When it moves for some row of the warp, the
+          // warp rescales its rows of O_s and its sums.  Only the item's own rows vote: a lane beyond them multiplies
+          // zero queries with whatever the slot holds.
+          auto new_reference = [&](float mx) {
+            const float cand = mx * scale;
+            if (!__any_sync(0xffffffffu, r < R && cand > m + kRescaleStep)) return;
+            const float mnew = fmaxf(m, cand);
+            const float alpha = m == -INFINITY ? 0.f : exp2f(m - mnew);
+            if (!own_first) scale_o(alpha);
+            l *= alpha;
+            m = mnew;
+          };
+          float lt = 0.f;
+          bool from_memory = false;
+          if (interior) {
+            // The stream's first tile of an item, or a row of the warp that has seen no key so far: references first.
+            // Pass 1 takes the row maxima (two chunks of 32 scores at a time) and moves the references.
+            const bool careful = own_first || __any_sync(0xffffffffu, r < R && m == -INFINITY);
+            float ya[32], yb[32];
+            if (careful) {
+              if (!p_waited && !wait_p()) { ok = false; break; }      // (the references may move, and O_s with them)
+              p_waited = true;
+              float mx = -INFINITY;
+              tmem_ld32(s_addr + 1 * 32, ya);
+              tmem_ld32(s_addr + 2 * 32, yb);
+              tmem_wait_ld();
+              mx = max32(max32(mx, ya), yb);
+              tmem_ld32(s_addr + 3 * 32, ya);
+              tmem_ld32(s_addr + 0 * 32, yb);
+              tmem_wait_ld();
+              mx = max32(max32(mx, ya), yb);
+              new_reference(mx);
+            }
+            // The weights, optimistically against the references as they stand: no maximum is taken.  The scores leave
+            // tensor memory for good before the last chunk's weights are computed, and the S buffer is released there.
+            // (a row that still sees nothing measures against 0: it has no finite score)
+            const float mref = m == -INFINITY ? 0.f : m;
             const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-mref, -mref);
             uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-            // the load of the next 32 scores is in flight while the weights of these 32 are computed
-            float ybuf[2][32];
-            tmem_ld32(s_addr, ybuf[0]);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-              float* const y = ybuf[c & 1];
+            // The first two chunks' weights wait in registers for the P buffer: the PV product that last read it follows
+            // this stream's previous tile by the time of eight products, which the stream would otherwise spend idle.
+            uint32_t pka[16], pkb[16];
+            tmem_ld32(s_addr + 0 * 32, yb);
+            tmem_ld32(s_addr + 3 * 32, ya);
+            tmem_wait_ld();
+            chunk_pack(yb, sc2, nm2, acc, pka);
+            tmem_ld32(s_addr + 1 * 32, yb);
+            chunk_pack(ya, sc2, nm2, acc, pkb);
+            tmem_wait_ld();
+            tmem_ld32(s_addr + 2 * 32, ya);
+            if (!p_waited && !wait_p()) { ok = false; break; }
+            tmem_st16u(p_addr + 0 * 16, pka);
+            tmem_st16u(p_addr + 3 * 16, pkb);
+            chunk_weights(1, yb, sc2, nm2, acc);
+            tmem_wait_ld();
+            release_s();
+            chunk_weights(2, ya, sc2, nm2, acc);
+            tmem_wait_st();
+            float s0, s1;
+            unpack2(add2(add2(acc[0], acc[1]), add2(acc[2], acc[3])), s0, s1);
+            lt = s0 + s1;
+            if (!careful) {
+              // A score far above its reference shows in the sum of the tile's weights (so does an overflow), and the
+              // test on the sum costs nothing per key.  Large but finite weights are as good as any (bf16 keeps their
+              // relative precision, O_s and the sum are fp32): the reference moves AFTERWARDS, to within 2^3.5 of the
+              // tile's maximum, the sum is rescaled now and the row of O_s at the stream's next tile, when this tile's
+              // PV product has completed.  Weights that may have overflowed are computed again from memory.
+              if (__any_sync(0xffffffffu, r < R && !(lt <= kGrowSum))) {
+                if (__any_sync(0xffffffffu, r < R && !(lt <= kHugeSum))) {
+                  from_memory = true;
+                } else {
+                  const float mnew = lt > kGrowSum ? m + log2f(lt) - 3.5f : m;
+                  o_alpha = exp2f(m - mnew);
+                  l = (l + lt) * o_alpha;
+                  lt = 0.f;
+                  m = mnew;
+                  o_owed = true;
+                }
+              }
+            }
+          } else {
+            // An item's last tile, a window's first: chunk by chunk.  A chunk that no row of the warp sees costs
+            // nothing (weights 0), one that every row sees in full runs unmasked, and only the chunks cut by some row's
+            // first or last key pay for the selects (rows beyond the item's own do not care).
+            auto chunk_class = [&](int c) -> int {          // 0: no row sees any key, 1: some row sees some, 2: all see all
+              const int t0 = t_first + c * 32;
+              if (__all_sync(0xffffffffu, r >= R || t0 > hi_r || t0 + 31 < lo_r)) return 0;
+              return __all_sync(0xffffffffu, r >= R || (t0 >= lo_r && t0 + 31 <= hi_r)) ? 2 : 1;
+            };
+            auto masked_scores = [&](int c, int cls, float* y) {
+              tmem_ld32(s_addr + c * 32, y);
               tmem_wait_ld();
-              if (c + 1 < NCH) tmem_ld32(s_addr + (c + 1) * 32, ybuf[(c + 1) & 1]);
-              uint32_t pk[16];
-              if constexpr (decltype(masked)::value) {
-                // Only the chunks that some row sees in part pay for masks: in an item's last tile most chunks lie
-                // wholly before every row's last key or wholly behind it (rows beyond the item's own do not care).
+              if (cls == 1) {
                 const int t0 = t_first + c * 32;
-                const bool none = __all_sync(0xffffffffu, r >= R || t0 > hi_r || t0 + 31 < lo_r);
-                if (none) {                               // no row of the warp sees any of these keys: weights 0
 #pragma unroll
-                  for (int e = 0; e < 16; ++e) pk[e] = 0u;
-                  tmem_st16u(p_addr + c * 16, pk);
-                  continue;
-                }
-                if (!__all_sync(0xffffffffu, r >= R || (t0 >= lo_r && t0 + 31 <= hi_r))) {
-#pragma unroll
-                  for (int e = 0; e < 32; ++e)
-                    if (t0 + e > hi_r || t0 + e < lo_r) y[e] = -INFINITY;
-                }
+                for (int e = 0; e < 32; ++e)
+                  if (t0 + e > hi_r || t0 + e < lo_r) y[e] = -INFINITY;
               }
+            };
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < NCH; ++c) {
+              const int cls = chunk_class(c);
+              if (cls == 0) continue;
+              float y[32];
+              masked_scores(c, cls, y);
+              mx = max32(mx, y);
+            }
+            new_reference(mx);
+            const float mref = m == -INFINITY ? 0.f : m;
+            const uint64_t sc2 = pack2(scale, scale), nm2 = pack2(-mref, -mref);
+            uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll 1
+            for (int c = 0; c < NCH; ++c) {
+              const int cls = chunk_class(c);
+              if (cls == 0) {
+                uint32_t pk[16];
 #pragma unroll
-              for (int e = 0; e < 32; e += 2) {
-                float d0, d1;
-                unpack2(fma2(pack2(y[e], y[e + 1]), sc2, nm2), d0, d1);
-                const float p0 = exp2f(d0), p1 = exp2f(d1);
-                acc[(e >> 1) & 3] = add2(acc[(e >> 1) & 3], pack2(p0, p1));
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+                for (int e = 0; e < 16; ++e) pk[e] = 0u;
+                tmem_st16u(p_addr + c * 16, pk);
+                continue;
               }
-              tmem_st16u(p_addr + c * 16, pk);            // 32 keys = 16 columns of the row's lane
+              float y[32];
+              masked_scores(c, cls, y);
+              chunk_weights(c, y, sc2, nm2, acc);
             }
             tmem_wait_st();
             float s0, s1;
             unpack2(add2(add2(acc[0], acc[1]), add2(acc[2], acc[3])), s0, s1);
-            return s0 + s1;
-          };
-
-          // Optimistic pass against the current references.  No maximum is tracked: a score more than 2^9 above its
-          // reference shows in the tile's sum of weights (so does an overflow), and the test on the sum costs
-          // nothing per key.  An item's first tile, and a tile that finds a row of the warp still without a
-          // reference (it has seen no key so far: sliding windows, split pairs), go straight to the careful pass.
-          // (only the item's own rows vote: a row beyond them multiplies zero queries with whatever the slot holds
-          // past the last key, and the result must not depend on that)
-          bool redo = own_first || __any_sync(0xffffffffu, r < R && m == -INFINITY);
-          float lt = 0.f;
-          if (!redo) {
-            lt = interior ? weights(m, std::false_type{}) : weights(m, std::true_type{});
-            redo = __any_sync(0xffffffffu, r < R && !(lt <= kRescaleSum));
+            lt = s0 + s1;
           }
-          if (redo) {
-            // some row of the warp outgrew its reference (or has none yet): every row of the warp takes its tile
-            // maximum, moves its reference, rescales its row of O_s and its sum, and computes its weights again
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-              float y[32];
-              if (interior) {
-                scores(c, y, std::false_type{});
-              } else {
-                // (chunk by chunk, as in the weights: nothing to do for a chunk that no row of the warp sees)
-                const int t0 = t_first + c * 32;
-                if (__all_sync(0xffffffffu, r >= R || t0 > hi_r || t0 + 31 < lo_r)) continue;
-                scores(c, y, std::true_type{});
-              }
-#pragma unroll
-              for (int e = 0; e < 32; ++e) mx = fmaxf(mx, y[e]);
-            }
-            const float mnew = fmaxf(m, mx * scale);
-            const float alpha = m == -INFINITY ? 0.f : exp2f(m - mnew);
-            if (!own_first) {
-              // O_s holds the products up to the stream's previous tile g - NS
-              if (NP != NS && !mbar_wait_c(bar_slot_empty((g - NS) % kSlots), ((g - NS) / kSlots) & 1u, ctl, P.status, 11)) { ok = false; break; }
-              tc_fence_after();
-#pragma unroll
-              for (int c = 0; c < D / 32; ++c) {
-                float o[32];
-                tmem_ld32(tmem_os + lane_addr + c * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) o[e] *= alpha;
-                tmem_st32(tmem_os + lane_addr + c * 32, o);
-              }
-              tmem_wait_st();
-            }
-            l *= alpha;
-            m = mnew;
-            // (a row that still sees nothing measures against 0: its masked keys get weight 2^-inf = 0)
-            lt = interior ? weights(m == -INFINITY ? 0.f : m, std::false_type{}) : weights(m == -INFINITY ? 0.f : m, std::true_type{});
+          if (from_memory) {
+            const int jm = r < R ? j : -1;
+            rows_tile_from_memory<D>(jm >= 0 ? A.q + ((size_t)(v.cu_q + jm / G) * P.Hq + v.kv_head * G + jm % G) * D : nullptr, A.k_pool,
+                                     A.block_table + (size_t)v.req * P.max_blocks, P.bs, P.Hkv, v.kv_head, P.num_blocks, kbase,
+                                     v.key_end, hi_r, lo_r, scale, p_addr, tmem_os + lane_addr, own_first, m, l);
+            lt = 0.f;
           }
           l += lt;
+        } else if (!wait_p()) {
+          // (a warp without rows announces P(g) too, and may do so only when the buffer's last reader is done:
+          // otherwise its arrival could land in the barrier's previous phase)
+          ok = false;
+          break;
         }
         own_first = false;
+        if (!s_released) release_s();
         tc_fence_before();
-        warp_arrive(bar_s_free(sbuf));
-        if (kbase + r >= v.key_end) {
+        if (kbase + rp >= v.key_end) {
           // keys past the end of the request: their V rows (page tail or a slot row that no copy touched) may
-          // hold anything, and 0 * NaN would poison O.  Zero them before the product.
-          const int vslot = g % kSlots;
-          if (mbar_wait_c(bar_slot_full(vslot), (g / kSlots) & 1u, ctl, P.status, 12)) {
-            unsigned char* vr = smem + vslot * L::kSlotBytes + v_off + (r >> 3) * SBO_KV + (r & 7) * 128;
+          // hold anything, and 0 * NaN would poison O.  Zero them before the product.  (Thread rp looks after key rp.)
+          const int vslot = g % VS;
+          if (mbar_wait_c(bar_v_full(vslot), (g / VS) & 1u, ctl, P.status, 12)) {
+            unsigned char* vr = smem + L::kOffV + vslot * L::kTileBytes + (rp >> 3) * SBO_KV + (rp & 7) * 128;
 #pragma unroll
             for (int x = 0; x < 8; ++x) *reinterpret_cast<uint4*>(vr + x * 16) = make_uint4(0, 0, 0, 0);
+            fence_proxy_async();
           }
         }
-        fence_proxy_async();
         warp_arrive(bar_p_full(pbuf));
         if (q_pending) {                                    // after the stream's first tile of the block: they have landed
           load_q_finish(item_idx + 1);
@@ -572,24 +839,39 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
       if (q_pending) load_q_finish(item_idx + 1);         // (a block in which this stream had no tile)
 
       // ---- epilogue: merge the streams' (m, l, O_s) of every row; thread (stream, r) finishes D / NS columns of row r ----
+      if (!mbar_wait_c(bar_o_full, item_idx & 1u, ctl, P.status, 13)) { ok = false; break; }
+      tc_fence_after();
+      if (o_owed) {
+        // the reference of some row moved after the stream's last tile: its row of O_s has yet to follow
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          float o[32];
+          tmem_ld32(tmem_os + lane_addr + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] *= o_alpha;
+          tmem_st32(tmem_os + lane_addr + c * 32, o);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+      }
       float2* const ml = ml_all + (item_idx & 1u) * (NS * L::kRows);
-      ml[stream * L::kRows + r] = make_float2(m, l);
+      ml[stream * L::kRows + rp] = make_float2(m, l);
       warp_arrive(bar_ml);
       if (!mbar_wait_c(bar_ml, item_idx & 1u, ctl, P.status, 14)) { ok = false; break; }
-      if (!mbar_wait_c(bar_o_full, item_idx & 1u, ctl, P.status, 13)) { ok = false; break; }
       tc_fence_after();
       if (warp_active) {
         constexpr int DC = D / NS;                          // output columns per thread
         float mt = -INFINITY;
 #pragma unroll
-        for (int t = 0; t < NS; ++t) mt = fmaxf(mt, ml[t * L::kRows + r].x);
+        for (int t = 0; t < NS; ++t) mt = fmaxf(mt, ml[t * L::kRows + rp].x);
         float lt = 0.f;
         float o[DC];
 #pragma unroll
         for (int e = 0; e < DC; ++e) o[e] = 0.f;
 #pragma unroll
         for (int t = 0; t < NS; ++t) {
-          const float2 x = ml[t * L::kRows + r];
+          const float2 x = ml[t * L::kRows + rp];
           const float wt = x.x == -INFINITY ? 0.f : exp2f(x.x - mt);
           lt = fmaf(wt, x.y, lt);
           float ot[DC];
@@ -649,13 +931,13 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kvmap, DevPlan P, AttnArgs 
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == L::kWarpMma) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
 
-cudaError_t launch_rows_instance(const CUtensorMap& kvm, const DevPlan& P, const AttnArgs& A, cudaStream_t s) {
+cudaError_t launch_rows_instance(const CUtensorMap& km, const CUtensorMap& vm, const DevPlan& P, const AttnArgs& A, cudaStream_t s) {
   constexpr int D = 64, NS = 2;
   const int smem = RowsSmem<D, NS>::kTotal + 1024;
   // the opt-in to large dynamic shared memory is per device and costs a few microseconds: once is enough
@@ -668,6 +950,6 @@ cudaError_t launch_rows_instance(const CUtensorMap& kvm, const DevPlan& P, const
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) opted_in[dev] = true;
   }
-  attn_rows_kernel<D, NS><<<A.num_ctas, RowsSmem<D, NS>::kThreads, smem, s>>>(kvm, P, A);
+  attn_rows_kernel<D, NS><<<A.num_ctas, RowsSmem<D, NS>::kThreads, smem, s>>>(km, vm, P, A);
   return cudaGetLastError();
 }

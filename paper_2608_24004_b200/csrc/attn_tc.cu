@@ -36,7 +36,6 @@
 #include "tc_ptx.cuh"
 
 namespace asv {
-
 namespace {
 
 constexpr int kTile = kTileKeys;                 // 128 keys per tile
@@ -334,11 +333,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 #pragma unroll
       for (int i = 0; i < SPW; ++i) {                     // every warpgroup stages the rows of its own slabs
         const int col0 = (wg + i * NWG) * 16;
-        const int rows_here = min(16, R - col0);
+        // (a slab that the item fills only in part gets zeros for the rest: what an earlier, wider item left there
+        // would otherwise vote on the references with scores that depend on bytes past the request's last key)
+        const int rows_here = col0 < R ? 16 : 0;
         for (int x = st; x < rows_here * CPR; x += 128) {
           const int row = col0 + x / CPR, ch = x % CPR;
-          const uint4 val = *reinterpret_cast<const uint4*>(
-              A.q + ((size_t)(v.cu_q + row / G) * P.Hq + v.kv_head * G + row % G) * D + ch * 8);
+          const uint4 val = row < R ? *reinterpret_cast<const uint4*>(
+              A.q + ((size_t)(v.cu_q + row / G) * P.Hq + v.kv_head * G + row % G) * D + ch * 8) : make_uint4(0, 0, 0, 0);
           *reinterpret_cast<uint4*>(qs + (ch / 8) * (NPAD * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = val;
         }
       }
@@ -359,12 +360,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 #pragma unroll
       for (int i = 0; i < SPW; ++i) {
         const int col0 = (wg + i * NWG) * 16;
-        const int rows_here = min(16, R - col0);
+        const int rows_here = col0 < R ? 16 : 0;            // (zeros behind the item's last row: see load_q)
         for (int x = st; x < rows_here * CPR; x += 128) {
           const int row = col0 + x / CPR, ch = x % CPR;
-          const __nv_bfloat16* src = A.q + ((size_t)(v.cu_q + row / G) * P.Hq + v.kv_head * G + row % G) * D + ch * 8;
           const uint32_t dst = qs + (ch / 8) * (NPAD * 128) + row * 128 + (((ch & 7) ^ (row & 7)) << 4);
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+          if (row < R) {
+            const __nv_bfloat16* src = A.q + ((size_t)(v.cu_q + row / G) * P.Hq + v.kv_head * G + row % G) * D + ch * 8;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+          } else {
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+          }
         }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
@@ -410,7 +415,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
             int jj = col0 / G, rem = col0 - jj * G;
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              if (t > v.n + jj || (W > 0 && t < v.n + jj - W + 1)) y[e] = -INFINITY;
+              if (t > v.n + jj || (W > 0 && t < v.n + jj - W + 1) || t >= v.key_end) y[e] = -INFINITY;
               if (++rem == G) {
                 rem = 0;
                 ++jj;
@@ -451,6 +456,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
               }
               lp[h * 8 + e] = fmaf(sign, p0, lp[h * 8 + e]);
               lp[h * 8 + e + 1] = fmaf(sign, p1, lp[h * 8 + e + 1]);
+              if (sign < 0.f) {
+                // a weight that overflowed cannot be taken back out (inf - inf); its reference is about to rise by
+                // 2^120 or more, which leaves nothing of the old partial sum anyway
+                if (!(fabsf(lp[h * 8 + e]) < INFINITY)) lp[h * 8 + e] = 0.f;
+                if (!(fabsf(lp[h * 8 + e + 1]) < INFINITY)) lp[h * 8 + e + 1] = 0.f;
+              }
               const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
               packed[e >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
             }
@@ -760,19 +771,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // so that one box = one (page, head) tile, delivered as 1024-byte atoms (8 rows x 128 bytes,
 // 128-byte swizzled) ordered [row group][row half]: the canonical shared-memory layout of a
 // tcgen05 operand with an 8-row-group stride of (D/64)*1024 bytes.
-// `kv_delta` = 0: the map covers one pool.  `kv_delta` > 0 (head_dim 64 only, where the row-half
-// dimension is free): that dimension selects between the two pools, `kv_delta` bytes apart, so one box
-// brings the K tile and the V tile of a (page, head) in a single copy, interleaved per 8-row group.
-bool encode_pool_map(void* map, const void* pool, int num_blocks, int Hkv, int bs, int D, uint64_t kv_delta,
-                     std::string& err) {
+bool encode_pool_map(void* map, const void* pool, int num_blocks, int Hkv, int bs, int D, std::string& err) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) {
     err = "cuTensorMapEncodeTiled is not available from the driver";
     return false;
   }
-  const cuuint64_t halves = kv_delta ? 2 : (cuuint64_t)(D / 64);
+  const cuuint64_t halves = (cuuint64_t)(D / 64);
   const cuuint64_t dims[5] = {64, 8, halves, (cuuint64_t)(bs / 8), (cuuint64_t)num_blocks * Hkv};
-  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, kv_delta ? kv_delta : 128, (cuuint64_t)8 * D * 2, (cuuint64_t)bs * D * 2};
+  const cuuint64_t strides[4] = {(cuuint64_t)D * 2, 128, (cuuint64_t)8 * D * 2, (cuuint64_t)bs * D * 2};
   const cuuint32_t box[5] = {64, 8, (cuuint32_t)halves, (cuuint32_t)(bs / 8), 1};
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   const CUresult r = fn(reinterpret_cast<CUtensorMap*>(map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5,
@@ -835,29 +842,16 @@ int launch_attn_tc(const DevPlan& P, const AttnArgs& A, TcState& st, cudaStream_
   if (A.num_ctas == 0) return 0;
   AttnArgs B = A;
   if (st.k_pool != A.k_pool || st.v_pool != A.v_pool) {
-    if (P.D == 64) {
-      // one map over both pools: the lower pool is the base, the other sits kv_delta bytes above it
-      const uintptr_t ka = reinterpret_cast<uintptr_t>(A.k_pool), va = reinterpret_cast<uintptr_t>(A.v_pool);
-      const uint64_t delta = ka < va ? va - ka : ka - va;
-      if (delta == 0 || (delta & 15) || delta >= (1ull << 40)) {
-        err = "head_dim 64 needs distinct K and V pools, 16-byte aligned and less than 2^40 bytes apart";
-        return 2;
-      }
-      if (!encode_pool_map(st.k_map, ka < va ? A.k_pool : A.v_pool, P.num_blocks, P.Hkv, P.bs, P.D, delta, err)) return 4;
-      std::memcpy(st.v_map, st.k_map, sizeof st.k_map);
-    } else {
-      if (!encode_pool_map(st.k_map, A.k_pool, P.num_blocks, P.Hkv, P.bs, P.D, 0, err)) return 4;
-      if (!encode_pool_map(st.v_map, A.v_pool, P.num_blocks, P.Hkv, P.bs, P.D, 0, err)) return 4;
-    }
+    if (!encode_pool_map(st.k_map, A.k_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
+    if (!encode_pool_map(st.v_map, A.v_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
     st.k_pool = A.k_pool;
     st.v_pool = A.v_pool;
   }
-  B.fused_k_first = reinterpret_cast<uintptr_t>(A.k_pool) < reinterpret_cast<uintptr_t>(A.v_pool) ? 1 : 0;
   const CUtensorMap& km = *reinterpret_cast<const CUtensorMap*>(st.k_map);
   const CUtensorMap& vm = *reinterpret_cast<const CUtensorMap*>(st.v_map);
   // the instance is as wide as this step's longest draft needs, not as the plan's maximum allows
   const int rows = A.rows_step > 0 ? A.rows_step : (P.Hq / P.Hkv) * (P.max_draft + 1);
-  const cudaError_t e = attn_rows_on_m(P.D, rows) ? launch_rows_instance(km, P, B, s) : launch_for_rows<128>(rows, km, vm, P, B, s);
+  const cudaError_t e = attn_rows_on_m(P.D, rows) ? launch_rows_instance(km, vm, P, B, s) : launch_for_rows<128>(rows, km, vm, P, B, s);
   if (e != cudaSuccess) {
     err = std::string("tensor-core attention launch: ") + cudaGetErrorString(e);
     return 4;

@@ -27,7 +27,6 @@ struct AttnArgs {
   int32_t num_ctas, num_merges;   // host side: grid sizes
   const int32_t* num_merges_dev;  // the step's merge count, in the workspace
   int32_t rows_step = 0;       // host side: most query rows any (request, kv-head) has in this step; picks the tile width
-  int32_t fused_k_first = 1;   // head_dim 64, tensor-core kernel: K pool lies below the V pool in memory
 };
 
 struct AcceptArgs {

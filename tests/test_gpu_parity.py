@@ -3,7 +3,7 @@
 Tolerances (written where they are applied): KV commit / rollback and greedy acceptance are
 bit-exact; attention output max-abs <= 2e-2 and mean-abs <= 2e-3 (plus, because those absolute bounds
 are about the size of the signal at long context, relative Frobenius error <= 1e-2 and
-|lse - lse*| <= 2e-3); sampled accept decisions exact except where the oracle's min(1, p/q) lies within
+|lse - lse*| <= 1e-3); sampled accept decisions exact except where the oracle's min(1, p/q) lies within
 1e-5 of the uniform (those positions are counted and must stay under 1e-4 of positions).
 """
 import math
@@ -18,7 +18,7 @@ from helpers import np_bits, oracle_attn, oracle_accept, oracle_commit, gather_l
 
 pytestmark = pytest.mark.gpu
 
-ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_FRO, LSE_ABS = 2e-2, 2e-3, 1e-2, 2e-3
+ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_FRO, LSE_ABS = 2e-2, 2e-3, 1e-2, 1e-3
 
 
 @pytest.fixture(scope="module")
@@ -146,8 +146,8 @@ def _random_shape(seed):
     Hkv = int(rng.choice([1, 2, 4, 8]))
     G = int(rng.choice([1, 2, 4, 8]))
     bs = int(rng.choice([16, 32, 64, 128]))
-    max_rows = 144 if D == 64 else 96
-    kmax = int(rng.integers(0, min(16, max_rows // G - 1) + 1))
+    max_rows = 256 if D == 64 else 128
+    kmax = int(rng.integers(0, min(31, max_rows // G - 1) + 1))
     window = int(rng.choice([0, 0, int(rng.integers(1, 400))]))
     B = int(rng.integers(1, 7))
     edges = np.array([0, 1, bs - 1, bs, bs + 1, 127, 128, 129, 255, 256, 257])
@@ -242,6 +242,84 @@ def test_needle_positions(bnd, impl_i):
                 got = out[j].float().cpu()
                 assert (got - want.float()[None, :]).abs().max() <= 2 ** -7 * want.float().abs().max() + 1e-6, (t, j)
         L.k_pool.copy_(kp); L.k_new.copy_(kn)
+
+
+def _scale_logical_pages(b, pool, factor_of_position):
+    """Multiplies the keys (or values) of every request's logical position t by factor_of_position(i, t) (a power of
+    two, so bf16 stays exact), page by page through the block table."""
+    bs = b.block_size
+    for i in range(b.batch):
+        for p in range(-(-int(b.seq_lens[i]) // bs)):
+            f = factor_of_position(i, p * bs)
+            if f != 1.0:
+                pool[b.block_table[i, p]] = (pool[b.block_table[i, p]].float() * f).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("impl_i", [0, 1])
+@pytest.mark.parametrize("D,Hq,dl", [(64, 64, [16, 3, 9, 0]), (64, 16, [15, 7, 2, 0]), (128, 32, [8, 3, 0, 6])])
+@pytest.mark.parametrize("factors", [(8.0, 64.0), (1.0, 512.0), (0.125, 1.0)])
+def test_scores_that_outgrow_their_reference(bnd, impl_i, D, Hq, dl, factors):
+    """Keys whose scale jumps in the middle of the context: the later tiles' scores lie tens to thousands of log2 units
+    above (or, shrinking, below) the running reference the first tiles set.  Covers references that move after a
+    tile's weights were computed and weights that overflow fp32 before they do."""
+    seq = [3000, 700, 1400, 129]
+    b = workloads.make_batch("t", seed=77, seq_lens=seq, draft_lens=dl, num_q_heads=Hq, num_kv_heads=8, head_dim=D,
+                             vocab=8, with_logits=False)
+    f1, f2 = factors
+    cut = lambda i, t: f2 if t >= (2 * seq[i]) // 3 // 128 * 128 + 48 else (f1 if t >= seq[i] // 3 else 1.0)
+    _scale_logical_pages(b, b.layers[0].k_pool, cut)
+    r = run_attn(bnd, b, impls(bnd)[impl_i])
+    if r is None:
+        pytest.skip("tensor-core kernel does not cover this shape")
+    _, out, lse = r
+    want, want_lse = oracle_attn(b)
+    mx, mean, rel = attn_errors(out, want)
+    assert mx <= ATTN_MAX_ABS and mean <= ATTN_MEAN_ABS and rel <= ATTN_REL_FRO, (mx, mean, rel)
+    # (an lse of several hundred carries fp32 rounding of its own: 1e-3 absolute plus 2e-6 relative)
+    assert (np.abs(lse.double().cpu().numpy() - want_lse) <= LSE_ABS + 2e-6 * np.abs(want_lse)).all()
+
+
+@pytest.mark.parametrize("impl_i", [0, 1])
+@pytest.mark.parametrize("D,Hq,window", [(64, 64, 0), (64, 64, 128), (128, 32, 0), (128, 32, 128)])
+def test_slots_no_request_can_see_may_hold_anything(bnd, impl_i, D, Hq, window):
+    """A real cache is not initialised: the tail of a request's last page, pages that no request owns and slots of
+    rolled-back drafts hold whatever was there before.  Fill every such slot of both pools with NaN and Inf bit patterns:
+    output and lse must be what they are with finite tails, bit for bit, and match the oracle.  Lengths are chosen so
+    that n + k + 1 is neither a multiple of 128 nor of the page size; one request is long enough to be split."""
+    seq = [70, 397, 40000 + 5, 1027, 255]
+    dl = [3, 9, 5, 0, 6] if D == 128 else [3, 16, 5, 0, 11]
+    g = torch.Generator().manual_seed(3)
+    kinds = [workloads.LayerKind(window=window, sinks=torch.randn(Hq, generator=g))]
+    b = workloads.make_batch("t", seed=88, seq_lens=seq, draft_lens=dl, num_q_heads=Hq, num_kv_heads=8, head_dim=D,
+                             vocab=8, kinds=kinds, with_logits=False)
+    r = run_attn(bnd, b, impls(bnd)[impl_i])
+    if r is None:
+        pytest.skip("tensor-core kernel does not cover this shape")
+    _, out0, lse0 = r
+    out0, lse0 = out0.clone(), lse0.clone()
+    want, want_lse = oracle_attn(b)
+    check_attn(out0, lse0, want, want_lse)
+    # poison: every slot at a position >= n_i + k_i + 1 of a request's pages, and every page nobody owns
+    L = b.layers[0]
+    bs = b.block_size
+    owned = np.zeros(L.k_pool.shape[0], bool)
+    poison = torch.tensor([float("nan"), float("inf"), -float("inf"), float("nan")]).to(torch.bfloat16)
+    for i in range(b.batch):
+        end = int(b.seq_lens[i] + b.draft_lens[i] + 1)
+        pages = -(-end // bs)
+        owned[b.block_table[i, :pages]] = True
+        if end % bs:
+            for pool in (L.k_pool, L.v_pool):
+                tail = pool[b.block_table[i, pages - 1], :, end % bs:, :]
+                tail.copy_(poison[torch.arange(tail.numel()) % 4].reshape(tail.shape))
+    for pool in (L.k_pool, L.v_pool):
+        free = torch.as_tensor(np.nonzero(~owned)[0])
+        if len(free):
+            pool[free] = float("nan")
+    r = run_attn(bnd, b, impls(bnd)[impl_i])
+    _, out1, lse1 = r
+    assert torch.equal(out0.view(torch.int16), out1.view(torch.int16))
+    assert torch.equal(lse0.view(torch.int32), lse1.view(torch.int32))
 
 
 def _check_sampled(bnd, b, vs):
