@@ -1,8 +1,8 @@
 /*
  * as_verify.h - C ABI of the batched verification step of speculative decoding on one B200.
  *
- * The step this library implements is the one the paper states in Sec. 2.2 ("speculatively
- * generating multiple tokens and verifying them with the target model", lossless) and Sec. 3
+ * The step this library implements is the one the paper states in Sec. 2.2 (draft several tokens,
+ * verify them with the target model in one pass, lossless) and Sec. 3
  * (D(b) drafted tokens per step, a per-request rejection rate), fed by the per-request draft lengths
  * L_i that Sec. 4.2 / Eq. 3 / Algorithm 2 allocate: request i of a batch brings k_i >= 0 draft
  * tokens (a single chain) and the target model scores k_i + 1 positions in one batched pass.
@@ -19,7 +19,8 @@
  * Pointers marked "dev" are device pointers owned by the caller and must stay valid until the work
  * enqueued on `stream` has finished; pointers marked "host" are read before the call returns.
  * The library allocates no device memory: all scratch lives in the workspace the caller binds to
- * the plan.  All GPU work is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL =
+ * the plan (one exception, as_accept_greedy_static, keeps its scratch in a fixed array of the library's
+ * device image and needs no plan).  All GPU work is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL =
  * the default stream) and is asynchronous with respect to the host.  A plan must not be used from
  * two host threads at once; distinct plans are independent.  Faults found on the device (a page id
  * outside the pool, a draft token outside the vocabulary, a bounded wait that ran out) set bits in
@@ -114,7 +115,7 @@ AS_API int as_plan_set_attn_impl(as_plan_t* plan, int impl);
  * after every later as_plan() of the same plan: as_plan() itself stays outside the recording (it is host
  * work plus one copy on the stream).  Costs one copy of the full metadata capacity per step and some
  * blocks that exit at once; meant for small batches, where a step is bound by launch overhead.  The paper
- * has no counterpart (its speculation length "adapts per step", Sec. 4.2, which is what this keeps cheap).
+ * has no counterpart (Sec. 4.2 / Eq. 3 choose the draft lengths anew in every step, which is what this keeps cheap).
  * Takes effect at the next as_plan(). */
 AS_API int as_plan_set_fixed_launch(as_plan_t* plan, int on);
 
@@ -141,8 +142,8 @@ AS_API int as_plan(as_plan_t* plan, int batch, const int32_t* seq_lens, const in
  * written and draft lengths chosen on the device - and free_blocks is a DEVICE int32 [num_free] or NULL; only the
  * number of requests is a host value.  Needs fixed launches (as_plan_set_fixed_launch), so the whole step - this
  * call, as_verify_attn per layer, as_accept, as_kv_commit - can be recorded once in a CUDA graph and replayed step
- * after step with nothing read back by the host (the paper's speculation length "adapts per step", Sec. 4.2: the
- * lengths change, the recording does not).  The work list is the one as_plan() builds for the same lengths, entry
+ * after step with nothing read back by the host (Sec. 4.2 / Eq. 3: the draft lengths change from step to step, the
+ * recording does not).  The work list is the one as_plan() builds for the same lengths, entry
  * for entry (both use one cost model and one cutting rule).  What as_plan() rejects with an error code cannot be
  * reported that way here: lengths out of range, a request that needs more pages than max_blocks_per_req, more
  * rows or pages than the plan's capacity, or a free list that is too short raise AS_FLAG_BAD_PLAN in the status
@@ -151,8 +152,8 @@ AS_API int as_plan(as_plan_t* plan, int batch, const int32_t* seq_lens, const in
 AS_API int as_plan_device(as_plan_t* plan, int batch, const int32_t* seq_lens, const int32_t* draft_lens,
                    int32_t* block_table, const int32_t* free_blocks, int num_free, void* stream);
 
-/* Verify attention for layer flavour `kind` (reading: Sec. 2.2 gives only "verify with the target
- * model"; the mask is the causal chain that a single drafted continuation implies, Sec. 4.2).
+/* Verify attention for layer flavour `kind` (reading: Sec. 2.2 says no more than that the target
+ * model verifies the drafts; the mask is the causal chain that a single drafted continuation implies, Sec. 4.2).
  *   q: dev bf16 [total_q, Hq, D].  k_new, v_new: dev bf16 [total_q, Hkv, D], the K/V of the step's
  *   own tokens.  k_pool, v_pool: dev bf16 [num_blocks, Hkv, bs, D] (16-byte aligned), updated in
  *   place: row j of request i is first stored at position n_i + j (tentative append), then
@@ -164,7 +165,7 @@ AS_API int as_plan_device(as_plan_t* plan, int batch, const int32_t* seq_lens, c
 AS_API int as_verify_attn(as_plan_t* plan, int kind, const void* q, const void* k_new, const void* v_new, void* k_pool,
                    void* v_pool, const int32_t* block_table, void* out, float* lse, void* stream);
 
-/* Acceptance over the vocabulary (reading of "lossless" verification, Sec. 2.2; rejection rate of
+/* Acceptance over the vocabulary (reading of lossless verification, Sec. 2.2; rejection rate of
  * Sec. 3 = 1 - sum a_i / sum k_i).  Logit row j of request i judges draft j+1.
  *   logits: dev fp32 [total_q, ld], ld >= vocab.  draft_tokens: dev int32 [total_d].
  *   temperature: dev fp32 [batch] or NULL.  NULL or T_i <= 0: greedy, the draft must equal the
@@ -198,7 +199,7 @@ AS_API int as_accept_seeded(as_plan_t* plan, const float* logits, int64_t ld, in
  *   logits[r][v] = sum_h hidden[r][h] * weight[v][h]
  * is computed on the tensor cores tile by tile and every tile is reduced at once to the row's largest logit and its
  * lowest column, so the [total_q, vocab] logits are never written to memory; the decision is then as_accept()'s
- * greedy one (reading: Sec. 2.2 says only "verify with the target model"; the paper's Sec. 3 names the growth of the
+ * greedy one (reading: Sec. 2.2 says only that the target model verifies the drafts; the paper's Sec. 3 names the growth of the
  * verification cost with the number of drafted tokens, which at large batches is this projection).
  *   hidden: dev bf16 [rows, hidden_dim], row stride hidden_dim, row r = row r of as_accept's logits; it must hold
  *     total_q rows (with fixed launches: max_batch * (max_draft + 1) rows, readable, contents beyond total_q unused).
@@ -257,6 +258,9 @@ AS_API int64_t as_plan_launch_count(const as_plan_t* plan);
  *   accept_len: dev int32 [batch]; out_tokens: dev int32 [batch, max_draft + 1] (-1 padded).
  * Same rule and same results as as_accept() with temperature = NULL: a draft is accepted while it
  * equals the lowest-index maximum of its row (NaN never wins), then the extra token follows.
+ * cu_q is read on the device and is not trusted: a request whose entries do not describe between 0 and
+ * max_draft drafts inside rows [0, total_q) gets accept_len 0 and a row of -1 (this entry point has no
+ * status word to report it through); the other requests are unaffected and nothing is read out of range.
  * Work is enqueued on `stream` for the current device.  The first call on a device looks up the
  * array's device address (cudaGetSymbolAddress, with that device current); make that first call
  * outside any stream capture.  All calls on a device share the one array and it keeps the previous

@@ -557,8 +557,8 @@ int ov_philox_uniforms(uint64_t seed, uint64_t step, int B, const int32_t* draft
   return 0;
 }
 
-// The target model's last layer in front of the acceptance test (a reading: Sec. 2.2 says only "verify with the
-// target model"; its output layer is a plain projection of the final hidden state onto the vocabulary):
+// The target model's last layer in front of the acceptance test (a reading: Sec. 2.2 says only that the
+// target model verifies the drafts; its output layer is a plain projection of the final hidden state onto the vocabulary):
 // logits[r][v] = sum_h hidden[r][h] * weight[v][h], bf16 inputs widened exactly, fp64 sum in index order.
 int ov_lm_head(int rows, int H, int V, const uint16_t* hidden, const uint16_t* weight, double* logits, int threads) {
   if (rows < 0 || H < 1 || V < 1 || !hidden || !weight || !logits) return 1;

@@ -72,7 +72,8 @@ __device__ void fold_row(const AcceptArgs& A, int row, int lane, Best& b, float&
 }
 
 __global__ void __launch_bounds__(kStatThreads) row_stats_kernel(DevPlan P, AcceptArgs A) {
-  const int row = blockIdx.y, chunk = blockIdx.x;
+  // (one block per (row, chunk), numbered along x: the y dimension of a grid ends at 65535 and a plan may hold more rows)
+  const int row = blockIdx.x / A.chunks, chunk = blockIdx.x - row * A.chunks;
   if (row >= P.hdr->total_q) return;                 // the grid may be sized for the plan's maximum
   const int req = P.row_map[row].x;
   const float T = A.temperature ? A.temperature[req] : 0.f;
@@ -303,7 +304,7 @@ __device__ __forceinline__ double rec_den(const AcceptArgs& A, int i) {     // c
 
 // Recovery, step 1: softmax denominator of row a_i in fp64, one CTA per vocabulary chunk.
 __global__ void __launch_bounds__(kRecThreads) recover_den_kernel(DevPlan P, AcceptArgs A) {
-  const int i = blockIdx.y, chunk = blockIdx.x;
+  const int i = blockIdx.x / A.chunks, chunk = blockIdx.x - i * A.chunks;
   if (i >= P.hdr->batch) return;
   const int a = A.recover_row[i];
   if (a < 0) return;
@@ -335,7 +336,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_den_kernel(DevPlan P, Acc
 // of max(0, p - q).  A warp owns whole cells and walks them in strips of 128 entries, four entries per lane,
 // four strips' loads in flight; the sums do not depend on the launch shape.
 __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, AcceptArgs A) {
-  const int i = blockIdx.y, chunk = blockIdx.x;
+  const int i = blockIdx.x / A.chunks, chunk = blockIdx.x - i * A.chunks;
   if (i >= P.hdr->batch) return;
   const int a = A.recover_row[i];
   if (a < 0) return;
@@ -480,17 +481,17 @@ __global__ void recover_pick_kernel(DevPlan P, AcceptArgs A) {
 
 cudaError_t launch_accept(const DevPlan& P, const AcceptArgs& A, cudaStream_t s) {
   if (P.batch == 0) return cudaSuccess;
-  row_stats_kernel<<<dim3(A.chunks, P.total_q), kStatThreads, 0, s>>>(P, A);
+  row_stats_kernel<<<(unsigned)A.chunks * (unsigned)P.total_q, kStatThreads, 0, s>>>(P, A);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   decide_kernel<<<(P.batch + 3) / 4, 128, 0, s>>>(P, A);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (A.temperature) {
-    recover_den_kernel<<<dim3(A.chunks, P.batch), kRecThreads, 0, s>>>(P, A);
+    recover_den_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    recover_cells_kernel<<<dim3(A.chunks, P.batch), kRecThreads, 0, s>>>(P, A);
+    recover_cells_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     recover_pick_kernel<<<(P.batch + 3) / 4, 128, 0, s>>>(P, A);

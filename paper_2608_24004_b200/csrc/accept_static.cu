@@ -88,14 +88,21 @@ __global__ void __launch_bounds__(kThreads) static_row_argmax_kernel(Scratch* sc
 }
 
 // One warp per request, lane = draft position: longest prefix of drafts that equal their row's argmax.
-__global__ void static_decide_kernel(const Scratch* sc, int batch, int max_draft, int vocab,
+// cu_q comes from device memory and is not trusted: a request whose entries do not describe 0 <= k <= max_draft rows
+// inside [0, total_q) is answered with accept_len 0 and a row of -1 instead of being read.
+__global__ void static_decide_kernel(const Scratch* sc, int batch, int total_q, int max_draft, int vocab,
                                      const int32_t* __restrict__ cu_q, const int32_t* __restrict__ draft_tokens,
                                      int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens) {
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= batch) return;
-  const int row0 = cu_q[i], k = min(cu_q[i + 1] - row0 - 1, max_draft), d0 = row0 - i;   // cu_d[i] = cu_q[i] - i
+  const int row0 = cu_q[i], k = cu_q[i + 1] - row0 - 1, d0 = row0 - i;   // cu_d[i] = cu_q[i] - i
   int32_t* outs = out_tokens + (size_t)i * (max_draft + 1);
+  if (row0 < i || k < 0 || k > max_draft || (long long)row0 + k >= total_q) {
+    for (int j = lane; j <= max_draft; j += 32) outs[j] = -1;
+    if (lane == 0) accept_len[i] = 0;
+    return;
+  }
   int a = k;
   for (int j0 = 0; j0 < k && a == k; j0 += 32) {
     const int j = j0 + lane;
@@ -164,7 +171,7 @@ int as_accept_greedy_static(int batch, int total_q, int max_draft, const int32_t
   static_row_argmax_kernel<<<dim3(chunks, total_q), kThreads, 0, s>>>(sc, logits, ld, vocab, chunk, chunks);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(AS_ERR_CUDA, std::string("as_accept_greedy_static: launch: ") + cudaGetErrorString(e));
-  static_decide_kernel<<<(batch + 3) / 4, 128, 0, s>>>(sc, batch, max_draft, vocab, cu_q, draft_tokens, accept_len, out_tokens);
+  static_decide_kernel<<<(batch + 3) / 4, 128, 0, s>>>(sc, batch, total_q, max_draft, vocab, cu_q, draft_tokens, accept_len, out_tokens);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(AS_ERR_CUDA, std::string("as_accept_greedy_static: launch: ") + cudaGetErrorString(e));
   return AS_OK;

@@ -1,8 +1,9 @@
 """GPU parity at the full sizes of the named workloads, in the launch configuration bench.py times.
 
-Attention is compared on sampled requests (all rows and heads of each), which the oracle can
-compute in seconds from a compact copy of just their pages; acceptance and commit are compared in
-full.  Tolerances as in test_gpu_parity.py."""
+Attention is compared on every request of the bench workload and on at least sixteen (eight at the sweep points)
+of the others - always the shortest, the longest, the longest and the shortest draft - with all rows and heads of
+each, which the oracle computes in seconds from a compact copy of just their pages; acceptance and commit are
+compared in full.  Tolerances as in test_gpu_parity.py."""
 import numpy as np
 import pytest
 import torch
@@ -36,7 +37,7 @@ def test_qwen3_8b_full_step(bnd):
     vs = bnd.VerifyStep(b)
     vs.plan_step(); vs.attn(0); vs.accept()
     assert bnd.as_plan_check(vs.plan) == 0
-    _attn_on_samples(bnd, b, vs, 0, _sample_requests(b, 8, np.random.default_rng(0)))
+    _attn_on_samples(bnd, b, vs, 0, list(range(b.batch)))            # all 64 requests
     ref = oracle_accept(b)
     assert np.array_equal(vs.accept_len.cpu().numpy(), ref["accept_len"])
     assert np.array_equal(vs.out_tokens.cpu().numpy(), ref["out_tokens"])
@@ -63,9 +64,9 @@ def test_gpt_oss_20b_layer_pair(bnd, all_max):
     vs = bnd.VerifyStep(b)
     vs.plan_step(); vs.attn(0); vs.attn(1); vs.accept()
     assert bnd.as_plan_check(vs.plan) == 0
-    ids = _sample_requests(b, 4, np.random.default_rng(1))
+    ids = _sample_requests(b, 16, np.random.default_rng(1))
     _attn_on_samples(bnd, b, vs, 0, ids)
-    _attn_on_samples(bnd, b, vs, 1, ids[:3])
+    _attn_on_samples(bnd, b, vs, 1, ids)
     ref = oracle_accept(b)
     assert np.array_equal(vs.accept_len.cpu().numpy(), ref["accept_len"])
     assert np.array_equal(vs.out_tokens.cpu().numpy(), ref["out_tokens"])
@@ -77,7 +78,7 @@ def test_r1_distill_llama_8b_stochastic(bnd):
     vs = bnd.VerifyStep(b)
     vs.plan_step(); vs.attn(0); vs.accept()
     assert bnd.as_plan_check(vs.plan) == 0
-    _attn_on_samples(bnd, b, vs, 0, _sample_requests(b, 6, np.random.default_rng(2)))
+    _attn_on_samples(bnd, b, vs, 0, _sample_requests(b, 16, np.random.default_rng(2)))
     in_band, total, exact = _check_sampled(bnd, b, vs)
     assert in_band < max(1, 1e-4 * total), (in_band, total)
     assert exact >= 0.99 * b.batch, exact
@@ -89,4 +90,4 @@ def test_sweep_points(bnd, batch, k, ctx):
     vs = bnd.VerifyStep(b)
     vs.plan_step(); vs.attn(0)
     assert bnd.as_plan_check(vs.plan) == 0
-    _attn_on_samples(bnd, b, vs, 0, _sample_requests(b, 3 if ctx > 10000 else 6, np.random.default_rng(3)))
+    _attn_on_samples(bnd, b, vs, 0, _sample_requests(b, 8, np.random.default_rng(3)))

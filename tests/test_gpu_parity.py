@@ -490,6 +490,32 @@ def test_commit_rollback_and_page_assignment(bnd):
         bnd.as_plan(vs.plan, seq, dl, torch.as_tensor(want_table).cuda(), None)
 
 
+def test_commit_leaves_table_entries_beyond_the_step_alone(bnd):
+    """Pages a scheduler reserved further out in a request's block-table row are not the step's to release: commit
+    frees only logical pages in [ceil(n'/bs), ceil((n+k+1)/bs)) and leaves later entries where they are."""
+    b = workloads.make_batch("t", seed=12, seq_lens=[30, 170, 62], draft_lens=[5, 2, 8], num_q_heads=8, num_kv_heads=2,
+                             head_dim=64, vocab=8, block_size=16, with_logits=False, k_max=8)
+    need = -(-(b.seq_lens + b.draft_lens + 1) // 16)
+    used = set(int(x) for x in b.block_table.ravel() if x >= 0)
+    spare = [p for p in range(b.num_blocks) if p not in used]
+    assert len(spare) >= 4
+    b.block_table[0, need[0]:need[0] + 2] = spare[:2]           # live entries past request 0's and 2's last position
+    b.block_table[2, need[2]] = spare[2]
+    for a in ([0, 0, 0], [5, 1, 3], [2, 2, 8]):
+        vs = bnd.VerifyStep(b)
+        vs.plan_step()
+        vs.attn(0)
+        vs.accept_len.copy_(torch.as_tensor(np.array(a, np.int32)))
+        vs.commit()
+        assert bnd.as_plan_check(vs.plan) == 0
+        seq2, bt2, _, _, freed = oracle_commit(b, a)
+        assert np.array_equal(vs.seq_lens.cpu().numpy(), seq2)
+        assert np.array_equal(vs.block_table.cpu().numpy(), bt2)
+        assert list(bt2[0, need[0]:need[0] + 2]) == spare[:2] and bt2[2, need[2]] == spare[2]
+        assert np.array_equal(vs.freed.cpu().numpy()[:int(vs.freed_count.item())], freed)
+        assert not set(freed.tolist()) & set(spare)
+
+
 def test_device_faults_are_flagged_not_trapped(bnd):
     b = workloads.make_batch("t", seed=4, seq_lens=[40, 40], draft_lens=[2, 2], num_q_heads=8, num_kv_heads=2,
                              head_dim=128, vocab=64, block_size=16, k_max=2)

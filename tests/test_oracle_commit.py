@@ -37,6 +37,25 @@ def test_hand_worked_paging(a, n_new, freed_logical):
     assert np.array_equal(got_v, want_v)
 
 
+@pytest.mark.parametrize("a,freed_logical", [(0, [2]), (2, []), (5, [])])
+def test_table_entries_past_the_steps_pages_are_not_released(a, freed_logical):
+    """Which pages a rollback releases: only those the STEP held, i.e. logical pages in
+    [ceil(n'/bs), ceil((n+k+1)/bs)).  A scheduler may have reserved pages further out in the same block-table row
+    (here logical pages 3 and 4, beyond the step's last position 11): they are not the step's to give back, so they
+    stay in the table and never show up in the freed list, whatever is accepted."""
+    b = _hand_batch()
+    assert b.block_table.shape[1] >= 5 and (b.block_table[0, 3:5] == -1).all()
+    spare = [p for p in range(64) if p not in set(b.block_table[0, :3].tolist())][:2]
+    b.block_table[0, 3:5] = spare
+    before = b.block_table.copy()
+    seq, bt, kp, vp, freed = oracle_commit(b, [a])
+    assert list(seq) == [6 + a + 1]
+    assert list(freed) == [int(before[0, l]) for l in freed_logical]
+    assert list(bt[0, 3:5]) == spare
+    keep = math.ceil((6 + a + 1) / 4)
+    assert (bt[0, keep:3] == -1).all() and (bt[0, :keep] == before[0, :keep]).all()
+
+
 def test_scrub_zeroes_rejected_slots_in_held_pages_only():
     b = _hand_batch()
     seq, bt, kp, vp, freed = oracle_commit(b, [2], scrub=True)        # n' = 9: slot 0 of page 2 kept
