@@ -90,6 +90,93 @@ def lm_head_leg(bnd, vs, b, workload, steps):
             hidden, weight)
 
 
+def roofline_of(bnd, b, vs, kind, attn_ms):
+    """KV bytes every (request, kv-head) must read once, over the measured duration of the attention launch(es) of layer
+    kind `kind` (CUDA events recorded by the library around them), against the measured copy bandwidth."""
+    peak, peak_kind = measured_peaks()
+    kv_bytes = b.kv_bytes(kind)
+    achieved = kv_bytes / (attn_ms * 1e-3) / 1e9
+    stats = bnd.as_plan_stats(vs.plan, kind)
+    tc_kernel = "attn_tc" if b.head_dim == 128 else "attn_rows"
+    roofline = {"bound": "hbm", "kernel": tc_kernel if stats["impl"] == bnd.AS_ATTN_TC else "attn_simt",
+                "achieved": achieved, "peak": peak, "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS, "traffic": None,
+                "algorithmic_bytes_per_launch": kv_bytes, "avg_launch_ms": attn_ms,
+                "ctas": stats["num_ctas"], "items": stats["num_items"], "merged_pairs": stats["num_merges"]}
+    if roofline["kernel"] != "attn_simt":
+        roofline["traffic"] = ATTN_TC_DRAM_BYTES_PER_KV_BYTE[b.head_dim] * kv_bytes
+        roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch on a batch-16 slice (ncu), "
+                                    "divided by that launch's algorithmic KV bytes, times this batch's KV bytes")
+    return roofline
+
+
+def other_workload(bnd, label, b, dev, steps, target_ms=250.0):
+    """One more named workload under the same clock: whole steps (plan + attention of every layer kind + acceptance +
+    commit) timed with CUDA events over a region of about target_ms, and per layer kind the attention launch's own
+    duration and roofline, computed exactly like the headline's."""
+    vs = bnd.VerifyStep(b, device=dev)
+    n_kinds = len(b.kinds)
+    bt0, seq0 = vs.block_table.clone(), vs.seq_lens.clone()
+
+    def run(n, pairs=None):
+        for i in range(n):
+            vs.block_table.copy_(bt0); vs.seq_lens.copy_(seq0)
+            vs.plan_step()
+            for kind in range(n_kinds):
+                if pairs is not None:
+                    bnd.as_plan_set_profile_events(vs.plan, *pairs[i][kind])
+                vs.attn(kind)
+            vs.accept()
+            vs.commit(kind=n_kinds - 1)
+    run(3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); run(3); e1.record()
+    torch.cuda.synchronize()
+    n = int(min(2000, max(steps, round(target_ms / max(e0.elapsed_time(e1) / 3, 1e-3)))))
+    pairs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_kinds)] for _ in range(n)]
+    for row in pairs:
+        for a, c in row:
+            a.record(); c.record()
+    e0.record(); run(n, pairs); e1.record()
+    torch.cuda.synchronize()
+    bnd.as_plan_set_profile_events(vs.plan, None, None)
+    assert bnd.as_plan_check(vs.plan) == 0
+    ms_step = e0.elapsed_time(e1) / n
+    entry = {"config": dict(workload_config(b, b.name), label=label), "timed_steps": n, "ms_per_step": ms_step,
+             "value": b.total_d / (ms_step * 1e-3), "unit": UNIT, "layers": []}
+    for kind in range(n_kinds):
+        attn_ms = statistics.mean(row[kind][0].elapsed_time(row[kind][1]) for row in pairs)
+        entry["layers"].append({"kind": kind, "window": int(b.kinds[kind].window), "roofline": roofline_of(bnd, b, vs, kind, attn_ms)})
+    entry["roofline"] = entry["layers"][-1]["roofline"]
+    return entry
+
+
+def other_workloads(bnd, dev, headline, steps):
+    """The named workloads other than the headline's, one after the other (each is freed before the next is built)."""
+    makers = [
+        ("gpt_oss_20b: window-128 layer + full layer, batch 128", "gpt_oss_20b", lambda: workloads.gpt_oss_20b(device=dev, seed=3000)),
+        ("gpt_oss_20b with every request at k = 16 (136 query rows per KV head)", "gpt_oss_20b_all_k16",
+         lambda: workloads.gpt_oss_20b(device=dev, seed=3000, all_max=True)),
+        ("r1_distill_llama_8b: batch 256, k = 6, sampled acceptance", "r1_distill_llama_8b",
+         lambda: workloads.r1_distill_llama_8b(device=dev, seed=4000)),
+        ("qwen3_8b, only the requests with n >= 8192", "qwen3_8b_min_context_8192",
+         lambda: workloads.qwen3_8b(device=dev, seed=2000, min_context=8192)),
+        ("r1_distill_llama_8b, only the requests with n >= 8192", "r1_distill_llama_8b_min_context_8192",
+         lambda: workloads.r1_distill_llama_8b(device=dev, seed=4000, min_context=8192)),
+        ("qwen3_8b: batch 64 (the headline workload of the default run)", "qwen3_8b", lambda: workloads.qwen3_8b(device=dev, seed=2000)),
+    ]
+    out = []
+    for label, key, make in makers:
+        if key == headline:
+            continue
+        b = make()
+        out.append(other_workload(bnd, label, b, dev, steps))
+        out[-1]["config"]["workload"] = key
+        del b
+        torch.cuda.empty_cache()
+    return out
+
+
 def make_workload(name, device, seed_offset=0, batch=None, min_context=0):
     over = {"batch": batch} if batch else {}
     if name == "qwen3_8b":
@@ -330,8 +417,13 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size (profiling only)")
     ap.add_argument("--min-context", type=int, default=0,
                     help="keep only the workload's requests with at least this committed length (profiling only)")
-    ap.add_argument("--lm-head", action="store_true",
-                    help="also time as_accept_lm_head (output projection fused with greedy acceptance) on this batch's rows")
+    ap.add_argument("--lm-head", action="store_true", help="(the default now: kept so that old command lines still parse)")
+    ap.add_argument("--no-lm-head", action="store_true",
+                    help="skip as_accept_lm_head (output projection fused with greedy acceptance) on this batch's rows")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the other named workloads (GPT-OSS-shaped pair, its all-k=16 variant, R1-shaped batch, n >= 8k subsets)")
+    ap.add_argument("--repeats", type=int, default=0, help="blocks of --steps steps inside the timed region (0: about --target-ms)")
+    ap.add_argument("--target-ms", type=float, default=1000.0, help="length of the timed region the repeats aim for")
     ap.add_argument("--sweep", action="store_true", help="run the batch x draft-length x context sweep instead")
     ap.add_argument("--sweep-out", default=None, help="markdown table of the sweep")
     args = ap.parse_args()
@@ -351,6 +443,7 @@ def main():
     from paper_2608_24004_b200 import build as as_build
     as_build.build_library()
     from paper_2608_24004_b200 import binding as bnd
+    from paper_2608_24004_b200 import replicas
 
     torch.cuda.set_device(local_rank)
     dist = None
@@ -375,8 +468,6 @@ def main():
         vs.accept()
         vs.commit(kind=n_kinds - 1)
 
-    from paper_2608_24004_b200 import replicas
-
     def barrier():
         replicas.barrier(dev)
 
@@ -384,30 +475,46 @@ def main():
         return replicas.max_over_ranks(ms, dev)
 
     # ---- device-resident timing -------------------------------------------------------------
+    # K = --steps steps form one block; the block is repeated R times back to back inside the timed region so that the
+    # region lasts about a second (the clock sampler then sees ten or more samples, and one slow step does not
+    # decide the number).  ms_per_step is the mean over all K * R steps; the per-block means give min / median / max.
     for _ in range(args.warmup):
         restore(); step()
     assert bnd.as_plan_check(vs.plan) == 0
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0.record()
+    for _ in range(3):
+        restore(); step()
+    w1.record()
+    torch.cuda.synchronize()
+    est_ms = max(w0.elapsed_time(w1) / 3, 1e-3)
+    repeats = args.repeats if args.repeats > 0 else int(min(400, max(1, round(args.target_ms / (est_ms * args.steps)))))
+    repeats = int(replicas.max_over_ranks(float(repeats), dev))
+    n_timed = args.steps * repeats
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_timed)]
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
     for a, c in pairs:
         a.record(); c.record()
     sampler = ClockSampler(local_rank)
     l0 = bnd.as_plan_launch_count(vs.plan)
     barrier()
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for a, c in pairs:
-        restore()
-        bnd.as_plan_set_profile_events(vs.plan, a, c)      # last layer kind of the step is the one kept
-        step()
-    e1.record()
+    marks[0].record()
+    for r in range(repeats):
+        for a, c in pairs[r * args.steps:(r + 1) * args.steps]:
+            restore()
+            bnd.as_plan_set_profile_events(vs.plan, a, c)      # last layer kind of the step is the one kept
+            step()
+        marks[r + 1].record()
     barrier()
     clocks = sampler.stop()
     bnd.as_plan_set_profile_events(vs.plan, None, None)
     launches = bnd.as_plan_launch_count(vs.plan) - l0
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
-    ms_step = ms_total / args.steps
-    attn_ms = statistics.mean(a.elapsed_time(c) for a, c in pairs)
+    ms_total = max_over_ranks(marks[0].elapsed_time(marks[-1]))
+    ms_step = ms_total / n_timed
+    block_ms = [marks[r].elapsed_time(marks[r + 1]) / args.steps for r in range(repeats)]
+    attn_all = [a.elapsed_time(c) for a, c in pairs]
+    attn_ms = statistics.mean(attn_all)
     assert bnd.as_plan_check(vs.plan) == 0
     total_drafts = replicas.sum_over_ranks(float(b.total_d), dev)
     value = total_drafts / (ms_step * 1e-3)
@@ -468,29 +575,18 @@ def main():
     assert int(h_acc.sum()) == int(vs.accept_len.sum())
 
     # ---- roofline of the dominant kernel (attention of the last layer kind) ----------------------
-    peak, peak_kind = measured_peaks()
-    kv_bytes = b.kv_bytes(n_kinds - 1)
-    achieved = kv_bytes / (attn_ms * 1e-3) / 1e9
-    stats = bnd.as_plan_stats(vs.plan, n_kinds - 1)
-    tc_kernel = "attn_tc" if b.head_dim == 128 else "attn_rows"
-    roofline = {"bound": "hbm", "kernel": tc_kernel if stats["impl"] == bnd.AS_ATTN_TC else "attn_simt",
-                "achieved": achieved, "peak": peak, "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS, "traffic": None,
-                "algorithmic_bytes_per_launch": kv_bytes, "avg_launch_ms": attn_ms,
-                "ctas": stats["num_ctas"], "items": stats["num_items"], "merged_pairs": stats["num_merges"]}
-    if roofline["kernel"] != "attn_simt":
-        roofline["traffic"] = ATTN_TC_DRAM_BYTES_PER_KV_BYTE[b.head_dim] * kv_bytes
-        roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch on a batch-16 slice (ncu --set full), "
-                                    "divided by that launch's algorithmic KV bytes, times the full batch's KV bytes")
+    roofline = roofline_of(bnd, b, vs, n_kinds - 1, attn_ms)
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "repeats": repeats, "timed_steps": n_timed, "timed_region_ms": ms_total,
+           "ms_per_step_blocks": {"min": min(block_ms), "median": statistics.median(block_ms), "max": max(block_ms)},
            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
            "data": "synthetic", "config": workload_config(b, args.workload), "clocks": clocks,
            "e2e": {"value": total_drafts / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
            "gpu_launches": int(launches), "roofline": roofline,
            "query_rows_per_s": b.total_q * world / (ms_step * 1e-3)}
-    if args.lm_head and rank == 0 and world == 1:
+    if not args.no_lm_head and rank == 0 and world == 1:
         lm, hidden, weight = lm_head_leg(bnd, vs, b, args.workload, max(3, min(args.steps, 10)))
         # the same end-to-end step with the hidden states as the step's input instead of the logits they project to
         # (the weights stay resident like the KV pools; greedy acceptance, whatever the workload's own mode)
@@ -526,6 +622,12 @@ def main():
             + pin_hidden.numel() * 2
         assert bnd.as_plan_check(vs.plan) == 0
         out["lm_head"] = lm
+    if rank == 0 and world == 1 and not args.no_other_workloads and not args.batch and not args.min_context:
+        del vs
+        if not args.no_lm_head:
+            del hidden, weight
+        torch.cuda.empty_cache()
+        out["other_workloads"] = other_workloads(bnd, dev, args.workload, max(3, min(args.steps, 10)))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         threads = oracle.hardware_threads()

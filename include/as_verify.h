@@ -238,6 +238,16 @@ AS_API int as_plan_set_profile_events(as_plan_t* plan, void* begin, void* end);
 /* Number of kernels this plan has launched since it was created (all calls, all streams). */
 AS_API int64_t as_plan_launch_count(const as_plan_t* plan);
 
+/* Test hook (no counterpart in the paper): exercises the bounded waits of the tensor-core attention kernels without
+ * any fault.  Every wait inside those kernels gives up after a time limit (2 s), raises AS_FLAG_WAIT_CAP plus a bit
+ * that names the wait, lets the CTA's other roles leave their loops, waits for copies in flight, frees its tensor
+ * memory and returns; as_plan_check() then reports AS_ERR_TIMEOUT.  This call shortens the limit to wait_limit_ns
+ * (0 = the default) and makes every CTA's copy producers stop issuing after stall_after_loads tile copies (-1 =
+ * never), so that the waits behind them run out.  The attention output of such a step is unspecified; nothing is
+ * read or written out of range, and the plan, the workspace and the device stay usable.  Applies to the following
+ * as_verify_attn calls of this plan until reset with (0, -1). */
+AS_API int as_plan_set_test_stall(as_plan_t* plan, uint64_t wait_limit_ns, int stall_after_loads);
+
 /* Greedy acceptance for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a convenience of the library, not part of the method.)
  *

@@ -24,7 +24,7 @@ AS_ATTN_AUTO, AS_ATTN_SIMT, AS_ATTN_TC = 0, 1, 2
 
 EXPORTS = ["as_status_string", "as_last_error", "as_plan_create", "as_plan_destroy", "as_plan_workspace_bytes",
            "as_plan_bind", "as_plan_set_attn_impl", "as_plan_set_fixed_launch", "as_plan", "as_plan_device", "as_verify_attn", "as_accept", "as_accept_seeded", "as_accept_lm_head", "as_kv_commit",
-           "as_plan_check", "as_plan_stats", "as_plan_preview", "as_plan_set_profile_events", "as_plan_launch_count", "as_budget",
+           "as_plan_check", "as_plan_stats", "as_plan_preview", "as_plan_set_profile_events", "as_plan_launch_count", "as_plan_set_test_stall", "as_budget",
            "as_accept_greedy_static", "as_drafter_create", "as_drafter_destroy", "as_drafter_open", "as_drafter_close", "as_drafter_forget",
            "as_drafter_feed", "as_drafter_block", "as_drafter_propose"]
 
@@ -62,6 +62,7 @@ def _load():
     lib.as_plan_set_profile_events.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.as_plan_launch_count.argtypes = [C.c_void_p]
     lib.as_plan_launch_count.restype = C.c_int64
+    lib.as_plan_set_test_stall.argtypes = [C.c_void_p, C.c_uint64, C.c_int]
     lib.as_budget.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_double, C.c_int, C.c_void_p,
                               C.c_void_p]
     lib.as_accept_greedy_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
@@ -264,6 +265,11 @@ def as_plan_set_profile_events(plan: Plan, begin=None, end=None):
 
 def as_plan_launch_count(plan: Plan) -> int:
     return int(_lib.as_plan_launch_count(plan.handle))
+
+
+def as_plan_set_test_stall(plan: Plan, wait_limit_ns: int = 0, stall_after_loads: int = -1):
+    """Test hook: shorter limit for the kernels' bounded waits, copy producers that stop after that many tiles."""
+    _chk(_lib.as_plan_set_test_stall(plan.handle, wait_limit_ns, stall_after_loads), "as_plan_set_test_stall")
 
 
 AS_STATIC_MAX_ROWS = 1024

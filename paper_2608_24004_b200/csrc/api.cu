@@ -95,6 +95,8 @@ struct as_plan_s {
   TcState tc;                 // tensor-map cache of the tensor-core kernel
   LmHeadState lm;             // tensor-map cache of the fused output projection
   cudaEvent_t prof_begin = nullptr, prof_end = nullptr;
+  unsigned long long test_wait_limit_ns = 0;   // as_plan_set_test_stall
+  int test_stall_after_loads = -1;
   int64_t launches = 0;
 };
 
@@ -665,6 +667,8 @@ int as_verify_attn(as_plan_t* p, int kind, const void* q, const void* k_new, con
   A.part_o = reinterpret_cast<float*>(p->ws + p->off_part_o);
   A.part_ml = reinterpret_cast<float2*>(p->ws + p->off_part_ml);
   A.num_ctas = st.num_ctas;
+  A.wait_limit_ns = p->test_wait_limit_ns;
+  A.stall_after_loads = p->test_stall_after_loads;
   if (p->prof_begin && p->prof_end) AS_CUDA(cudaEventRecord(p->prof_begin, s));
   for (int sb = 0; sb < st.num_sub; ++sb) {
     const SubLaunch& sl = st.sub[sb];
@@ -844,6 +848,13 @@ int as_plan_set_profile_events(as_plan_t* p, void* begin, void* end) {
 }
 
 int64_t as_plan_launch_count(const as_plan_t* p) { return p ? p->launches : 0; }
+
+int as_plan_set_test_stall(as_plan_t* p, uint64_t wait_limit_ns, int stall_after_loads) {
+  if (!p || stall_after_loads < -1) return fail(AS_ERR_INVALID_ARG, "as_plan_set_test_stall: bad argument");
+  p->test_wait_limit_ns = wait_limit_ns;
+  p->test_stall_after_loads = stall_after_loads;
+  return AS_OK;
+}
 
 int as_plan_preview(const as_plan_t* p, int kind, int num_ctas, int batch, const int32_t* seq_lens,
                     const int32_t* draft_lens, int32_t* items_out, int cap_items, int32_t* cta_first_out,

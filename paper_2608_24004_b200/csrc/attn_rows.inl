@@ -319,6 +319,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
     mbar_init(bar_ml, 4 * NS);
     ctl->abort = 0;
     ctl->tmem_base = 0;
+    ctl->limit_ns = A.wait_limit_ns ? A.wait_limit_ns : kWaitLimitNs;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int x = tid; x < min(it_end - it_begin, kItemCache) * 2; x += kThreads)
@@ -375,6 +376,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
         const int ids_next = c + 1 < nch ? chunk_load(v, c + 1) : (nit < it_end ? chunk_load(nv, 0) : -1);
         const int t_end = min(v.tiles, (c + 1) * tiles_per_chunk);
         for (int tile = c * tiles_per_chunk; tile < t_end; ++tile) {
+          if (A.stall_after_loads >= 0 && (int)load_idx >= A.stall_after_loads) { ok = false; break; }   // (test hook: the copies stop coming)
           const int kbase = v.key_begin + tile * kTile;
           const int npages = min(pages_per_tile, (v.key_end - kbase + P.bs - 1) / P.bs);
           int page = __shfl_sync(0xffffffffu, ids, ((tile - c * tiles_per_chunk) * pages_per_tile + lane) & 31);
@@ -482,7 +484,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
           const unsigned long long now = global_ns();
           if (idle_since == 0) {
             idle_since = now;
-          } else if (now - idle_since > kWaitLimitNs) {
+          } else if (now - idle_since > ctl->limit_ns) {
             ctl->abort = 1;
             atomicOr(P.status, kFlagWaitCap | (1u << (8 + 2)));
             break;

@@ -153,6 +153,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     for (int w = 0; w < NWG; ++w) mbar_init(bar_wg(w), 128);
     ctl->abort = 0;
     ctl->tmem_base = 0;
+    ctl->limit_ns = A.wait_limit_ns ? A.wait_limit_ns : kWaitLimitNs;
     for (int x = 0; x < 32; ++x) (&ctl->flags[0][0])[x] = 0;
     for (int x = 0; x < NPAD; ++x) wmax[x] = (int)0x807fffff;      // order-preserving image of -inf
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,6 +210,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         page = -1;
       }
       const int nvalid = __popc(__ballot_sync(0xffffffffu, page >= 0));
+      if (A.stall_after_loads >= 0 && (int)load_idx >= A.stall_after_loads) break;   // (test hook: the copies stop coming)
       for (int which = 0; which < 2; ++which) {
         const int slot = load_idx % kSlots;
         const uint32_t par = ((load_idx / kSlots) & 1u) ^ 1u;

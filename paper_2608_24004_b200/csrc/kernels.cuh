@@ -27,6 +27,10 @@ struct AttnArgs {
   int32_t num_ctas, num_merges;   // host side: grid sizes
   const int32_t* num_merges_dev;  // the step's merge count, in the workspace
   int32_t rows_step = 0;       // host side: most query rows any (request, kv-head) has in this step; picks the tile width
+  // test hooks of the tensor-core kernels (as_plan_set_test_stall): a shorter limit for the bounded waits, and a number of
+  // tile copies after which a CTA's producers stop issuing, so that the waits behind them run out
+  unsigned long long wait_limit_ns = 0;
+  int32_t stall_after_loads = -1;
 };
 
 struct AcceptArgs {

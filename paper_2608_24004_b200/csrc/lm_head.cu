@@ -66,6 +66,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap amap, const __grid_con
     }
     ctl->abort = 0;
     ctl->tmem_base = 0;
+    ctl->limit_ns = kWaitLimitNs;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {

@@ -45,6 +45,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 struct Ctl {                 // small control block in shared memory
   volatile int abort;
   uint32_t tmem_base;
+  unsigned long long limit_ns;  // how long a wait may last (kWaitLimitNs unless a test shortened it)
   uint32_t flags[8][4];      // per softmax warpgroup: three rotating "a score outgrew its reference" words (+ 1 pad)
 };
 
@@ -59,7 +60,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctl* ct
       const unsigned long long now = global_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > ctl->limit_ns) {
         ctl->abort = 1;
         atomicOr(status, kFlagWaitCap | (1u << (8 + site)));
         return false;

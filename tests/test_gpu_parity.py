@@ -535,6 +535,36 @@ def test_device_faults_are_flagged_not_trapped(bnd):
     assert float(out.sum()) == 4.0
 
 
+@pytest.mark.parametrize("D,Hq,stall", [(128, 32, 3), (128, 32, 0), (64, 64, 5), (64, 64, 0)])
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_plan_usable(bnd, D, Hq, stall):
+    """Failure detection without a fault: the test hook tells every CTA's copy producers to stop after `stall` tiles
+    and shortens the kernels' wait limit to 3 ms, so the waits behind the missing copies run out.  The kernel must
+    return by itself, as_plan_check must report AS_ERR_TIMEOUT with AS_FLAG_WAIT_CAP and a bit naming a wait, and the
+    next ordinary step on the same plan, workspace and pools must equal a step on a fresh plan bit for bit."""
+    b = workloads.make_batch("t", seed=21, seq_lens=[3000, 900, 5000, 129], draft_lens=[4, 8, 0, 6], num_q_heads=Hq,
+                             num_kv_heads=8, head_dim=D, vocab=8, with_logits=False)
+    fresh = bnd.VerifyStep(b, attn_impl=bnd.AS_ATTN_TC)
+    fresh.plan_step(); fresh.attn(0)
+    assert bnd.as_plan_check(fresh.plan) == 0
+    want_out, want_lse = fresh.out[0].clone(), fresh.lse[0].clone()
+
+    vs = bnd.VerifyStep(b, attn_impl=bnd.AS_ATTN_TC)
+    vs.plan_step()
+    bnd.as_plan_set_test_stall(vs.plan, 3_000_000, stall)
+    vs.attn(0)
+    with pytest.raises(bnd.AsError) as e:
+        bnd.as_plan_check(vs.plan)
+    assert e.value.status == bnd.AS_ERR_TIMEOUT
+    vs.plan_step(); vs.attn(0)                                 # still stalling: the flags say which waits gave up
+    flags = bnd.as_plan_check(vs.plan, raise_on_flag=False)
+    assert flags & bnd.AS_FLAG_WAIT_CAP and flags >> 8, hex(flags)
+    bnd.as_plan_set_test_stall(vs.plan, 0, -1)
+    vs.plan_step(); vs.attn(0)
+    assert bnd.as_plan_check(vs.plan) == 0
+    assert torch.equal(vs.out[0].view(torch.int16), want_out.view(torch.int16))
+    assert torch.equal(vs.lse[0].view(torch.int32), want_lse.view(torch.int32))
+
+
 def test_empty_batch_and_argument_errors(bnd):
     b = workloads.tiny()
     vs = bnd.VerifyStep(b)
