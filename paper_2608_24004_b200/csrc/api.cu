@@ -74,7 +74,6 @@ struct as_plan_s {
   as_layer_desc kinds[kMaxKinds];
   int max_batch = 0, max_draft = 0, max_blocks = 0, num_blocks = 0;
   int Hq = 0, Hkv = 0, D = 0, bs = 0, G = 0, rows_max = 0;
-  int rows_step = 0;             // G * (longest draft of the current step + 1), or rows_max with fixed launches
   int impl_request = AS_ATTN_AUTO;
   int simt_ctas_per_sm = 1;
   bool fixed_launch = false;     // lay the metadata out at fixed offsets and size every grid for the plan's maxima
@@ -139,18 +138,33 @@ void build_work(const as_plan_s* p, int kind, int impl, int P, int rows_inst, co
                 std::vector<WorkItem>& items, std::vector<int32_t>& cta_first, std::vector<MergeSeg>& merges) {
   const int W = p->kinds[kind].window;
   const bool rows_on_m = impl == AS_ATTN_TC && attn_rows_on_m(p->D, rows_inst);
-  std::vector<int32_t> t_first(batch), t_count(batch);
-  std::vector<int64_t> cpt(batch), ovh(batch);
+  // a request is one pair per kv-head, or - where the kernel holds fewer rows than the request has - one per block of
+  // draft positions (plan_block_positions): `Blk` is what the kernels see as a request
+  struct Blk {
+    int32_t req, n, k, cu_q, t_first, t_count;
+    int64_t cpt, ovh;
+  };
+  std::vector<Blk> blks;
   int64_t C = 0;
-  for (int i = 0; i < batch; ++i) {
-    const int end = seq[i] + dl[i] + 1;
-    const int lo = W > 0 ? std::max(0, seq[i] - W + 1) : 0;
-    t_first[i] = lo / kTileKeys;
-    t_count[i] = (end + kTileKeys - 1) / kTileKeys - t_first[i];
-    cpt[i] = plan_tile_cost(impl == AS_ATTN_TC, rows_on_m, rows_inst, p->G * (dl[i] + 1));
-    ovh[i] = plan_item_overhead(impl == AS_ATTN_TC, rows_on_m, p->G * (dl[i] + 1));
-    if (member && !member[i]) t_count[i] = -1;                       // not in this launch
-    else C += (ovh[i] + t_count[i] * cpt[i]) * p->Hkv;
+  int cu_q = 0;
+  for (int i = 0; i < batch; cu_q += dl[i] + 1, ++i) {
+    if (member && !member[i]) continue;                                // not in this launch
+    const int pb = plan_block_positions(impl == AS_ATTN_TC, rows_on_m, p->G, dl[i]);
+    for (int first = 0; first <= dl[i]; first += pb) {
+      Blk b;
+      b.req = i;
+      b.n = seq[i] + first;
+      b.k = std::min(dl[i] - first, pb - 1);
+      b.cu_q = cu_q + first;
+      const int end = b.n + b.k + 1;
+      const int lo = W > 0 ? std::max(0, b.n - W + 1) : 0;
+      b.t_first = lo / kTileKeys;
+      b.t_count = (end + kTileKeys - 1) / kTileKeys - b.t_first;
+      b.cpt = plan_tile_cost(impl == AS_ATTN_TC, rows_on_m, rows_inst, p->G * (b.k + 1));
+      b.ovh = plan_item_overhead(impl == AS_ATTN_TC, rows_on_m, p->G * (b.k + 1));
+      C += (b.ovh + b.t_count * b.cpt) * p->Hkv;
+      blks.push_back(b);
+    }
   }
   items.clear();
   merges.clear();
@@ -158,35 +172,33 @@ void build_work(const as_plan_s* p, int kind, int impl, int P, int rows_inst, co
   if (C == 0) return;
   std::vector<int32_t> owners;
   int64_t c0 = 0;
-  int cu_q = 0;
-  for (int i = 0; i < batch; cu_q += dl[i] + 1, ++i) {
-    if (t_count[i] < 0) continue;
-    const int R = p->G * (dl[i] + 1);
-    const int end = seq[i] + dl[i] + 1;
+  for (const Blk& b : blks) {
+    const int R = p->G * (b.k + 1);
+    const int end = b.n + b.k + 1;
     for (int g = 0; g < p->Hkv; ++g) {
       const size_t first_item = items.size();
       int parts = 0;
-      for (int t = 0, t_end, o; t < t_count[i]; t = t_end, ++parts) {
-        plan_next_piece(c0 + ovh[i], t, t_count[i], cpt[i], C, P, t_end, o);
+      for (int t = 0, t_end, o; t < b.t_count; t = t_end, ++parts) {
+        plan_next_piece(c0 + b.ovh, t, b.t_count, b.cpt, C, P, t_end, o);
         WorkItem w{};
-        w.req = i;
+        w.req = b.req;
         w.kv_head = g;
-        w.key_begin = (t_first[i] + t) * kTileKeys;
-        w.key_end = std::min(end, (t_first[i] + t_end) * kTileKeys);
+        w.key_begin = (b.t_first + t) * kTileKeys;
+        w.key_end = std::min(end, (b.t_first + t_end) * kTileKeys);
         w.part_row = -1;
-        w.n = seq[i];
-        w.k = dl[i];
-        w.cu_q = cu_q;
+        w.n = b.n;
+        w.k = b.k;
+        w.cu_q = b.cu_q;
         items.push_back(w);
         owners.push_back(o);
       }
       if (parts > 1) {
-        MergeSeg m{i, g, part_rows, parts};
+        MergeSeg m{b.req, g, part_rows, parts, b.k, b.cu_q};
         merges.push_back(m);
         for (int s = 0; s < parts; ++s) items[first_item + s].part_row = part_rows + s * R;
         part_rows += parts * R;
       }
-      c0 += ovh[i] + t_count[i] * cpt[i];
+      c0 += b.ovh + b.t_count * b.cpt;
     }
   }
   // cta_first[c] = first item owned by a CTA >= c
@@ -195,6 +207,29 @@ void build_work(const as_plan_s* p, int kind, int impl, int P, int rows_inst, co
     while (at < items.size() && owners[at] < c) ++at;
     cta_first[c] = (int32_t)at;
   }
+}
+
+// Row blocks a request can have at most under this plan (1 unless the keys-on-M kernel serves more than 128 rows).
+int max_row_blocks(const as_plan_s* p) {
+  if (p->D != 128) return 1;
+  int v = 1;
+  for (int k = 0; k <= p->max_draft; ++k) {
+    const int pb = plan_block_positions(true, false, p->G, k);
+    v = std::max(v, (k + pb) / pb);
+  }
+  return v;
+}
+
+// Most query rows a launch item of a request with k drafts has (the request's own, or its widest row block's).
+int item_rows(const as_plan_s* p, int impl, int k) {
+  const bool tc = impl == AS_ATTN_TC;
+  return p->G * std::min(k + 1, plan_block_positions(tc, tc && attn_rows_on_m(p->D, p->G * (k + 1)), p->G, k));
+}
+// ... of any request with up to kmax drafts: what picks the kernel instance of a launch.
+int launch_rows(const as_plan_s* p, int impl, int kmax) {
+  int rows = 0;
+  for (int k = 0; k <= kmax; ++k) rows = std::max(rows, item_rows(p, impl, k));
+  return rows;
 }
 
 }  // namespace
@@ -284,7 +319,7 @@ int as_plan_create(as_plan_t** out, const as_layer_desc* kinds, int num_kinds, i
   meta += align_up(sizeof(int2) * p->max_total_q, 16);
   meta += align_up(sizeof(int32_t) * (max_batch + 1), 16);
   meta += align_up(sizeof(int32_t) * p->max_free, 16);
-  const size_t max_items = (size_t)max_batch * p->Hkv + kMaxSub * p->max_ctas;
+  const size_t max_items = (size_t)max_batch * p->Hkv * max_row_blocks(p) + kMaxSub * p->max_ctas;
   for (int i = 0; i < num_kinds; ++i) {
     meta += align_up(sizeof(WorkItem) * max_items, 16);
     meta += kMaxSub * align_up(sizeof(int32_t) * (p->max_ctas + 1), 16);
@@ -383,7 +418,6 @@ int as_plan(as_plan_t* p, int batch, const int32_t* seq_lens, const int32_t* dra
   p->total_d = (int)td;
   int kmax_step = 0;
   for (int i = 0; i < batch; ++i) kmax_step = std::max(kmax_step, (int)draft_lens[i]);
-  p->rows_step = p->fixed_launch ? p->rows_max : p->G * (kmax_step + 1);
   char* hm = p->host_meta.data();
   size_t off = 0;
   // every array takes what this step needs, or - with fixed launches - its full capacity, so that its
@@ -393,7 +427,7 @@ int as_plan(as_plan_t* p, int batch, const int32_t* seq_lens, const int32_t* dra
     off += align_up(p->fixed_launch ? capacity : bytes, 16);
     return at;
   };
-  const size_t max_items = (size_t)p->max_batch * p->Hkv + kMaxSub * p->max_ctas;
+  const size_t max_items = (size_t)p->max_batch * p->Hkv * max_row_blocks(p) + kMaxSub * p->max_ctas;
   const size_t o_hdr = take(sizeof(StepHeader), sizeof(StepHeader));
   const size_t o_req = take(sizeof(ReqMeta) * batch, sizeof(ReqMeta) * p->max_batch);
   const size_t o_map = take(sizeof(int2) * tq, sizeof(int2) * p->max_total_q);
@@ -433,10 +467,11 @@ int as_plan(as_plan_t* p, int batch, const int32_t* seq_lens, const int32_t* dra
     // launch of like requests balances better).  Two classes at most; one when launches must be fixed, when
     // the step is small, or when a class would be nearly empty.
     std::vector<uint8_t> member[kMaxSub];
-    int rows_of[kMaxSub] = {p->rows_step};
+    const int rows_kind = launch_rows(p, st.impl, p->fixed_launch ? p->max_draft : kmax_step);
+    int rows_of[kMaxSub] = {rows_kind};
     st.num_sub = 1;
     // (the rows-on-M kernel's tile cost does not depend on the row count: nothing to gain there)
-    if (st.impl == AS_ATTN_TC && !p->fixed_launch && p->rows_step > kRowClassCut && !attn_rows_on_m(p->D, p->rows_step)) {
+    if (st.impl == AS_ATTN_TC && !p->fixed_launch && rows_kind > kRowClassCut && !attn_rows_on_m(p->D, rows_kind)) {
       int cuts[kMaxSub - 1];
       for (int c = 0; c < kMaxSub - 1; ++c) cuts[c] = 1 << 30;
       cuts[0] = kRowClassCut;
@@ -444,7 +479,7 @@ int as_plan(as_plan_t* p, int batch, const int32_t* seq_lens, const int32_t* dra
       int rows_max_of[kMaxSub] = {};
       std::vector<uint8_t> cls(batch);
       for (int i = 0; i < batch; ++i) {
-        const int R = p->G * (draft_lens[i] + 1);
+        const int R = item_rows(p, st.impl, draft_lens[i]);      // (a wide request counts by its row blocks)
         int c = 0;
         while (c < kMaxSub - 1 && R > cuts[c]) ++c;
         cls[i] = (uint8_t)c;
@@ -496,7 +531,7 @@ int as_plan(as_plan_t* p, int batch, const int32_t* seq_lens, const int32_t* dra
             member[slot_of[c]][i] = 1;
           }
         } else {
-          rows_of[0] = p->rows_step;
+          rows_of[0] = rows_kind;
         }
       }
     }
@@ -559,7 +594,6 @@ int as_plan_device(as_plan_t* p, int batch, const int32_t* seq_lens, const int32
   p->batch = batch;
   p->total_q = p->max_total_q;
   p->total_d = p->max_draft > 0 ? p->max_total_q : 0;   // (what as_accept's null check goes by: drafts are possible)
-  p->rows_step = p->rows_max;
   // the same fixed layout as_plan() uses with fixed launches: every array at its full capacity
   size_t off = 0;
   auto take = [&](size_t capacity) {
@@ -567,7 +601,7 @@ int as_plan_device(as_plan_t* p, int batch, const int32_t* seq_lens, const int32
     off += align_up(capacity, 16);
     return at;
   };
-  const size_t max_items = (size_t)p->max_batch * p->Hkv + kMaxSub * p->max_ctas;
+  const size_t max_items = (size_t)p->max_batch * p->Hkv * max_row_blocks(p) + kMaxSub * p->max_ctas;
   const size_t o_hdr = take(sizeof(StepHeader));
   const size_t o_req = take(sizeof(ReqMeta) * p->max_batch);
   const size_t o_map = take(sizeof(int2) * p->max_total_q);
@@ -591,7 +625,7 @@ int as_plan_device(as_plan_t* p, int batch, const int32_t* seq_lens, const int32
     st.num_ctas = st.impl == AS_ATTN_TC ? p->num_sms : p->num_sms * p->simt_ctas_per_sm;
     st.num_sub = 1;
     SubLaunch& sl = st.sub[0];
-    sl.rows_inst = p->rows_max;
+    sl.rows_inst = launch_rows(p, st.impl, p->max_draft);
     // counts stay on the device: the merge grid covers the capacity, the kernels read the step's counts
     sl.num_items = st.num_items = -1;
     sl.num_merges = st.num_merges = p->max_ctas;
@@ -607,6 +641,7 @@ int as_plan_device(as_plan_t* p, int batch, const int32_t* seq_lens, const int32
     K.rows_inst = sl.rows_inst;
     K.tensor_core = st.impl == AS_ATTN_TC;
     K.rows_on_m = K.tensor_core && attn_rows_on_m(p->D, sl.rows_inst);
+    K.row_blocks = K.tensor_core && !K.rows_on_m ? max_row_blocks(p) : 1;
   }
   if (off > p->meta_capacity) return fail(AS_ERR_WORKSPACE, "as_plan_device: metadata exceeds the planned capacity");
   a.G = p->G;
@@ -873,7 +908,7 @@ int as_plan_preview(const as_plan_t* p, int kind, int num_ctas, int batch, const
   int kmax_step = 0;
   for (int i = 0; i < batch; ++i) kmax_step = std::max(kmax_step, (int)draft_lens[i]);
   int part_rows = 0;
-  build_work(p, kind, impl, num_ctas, p->fixed_launch ? p->rows_max : p->G * (kmax_step + 1), seq_lens, draft_lens, batch,
+  build_work(p, kind, impl, num_ctas, launch_rows(p, impl, p->fixed_launch ? p->max_draft : kmax_step), seq_lens, draft_lens, batch,
              nullptr, part_rows, items, cta_first, merges);
   if (items_out)
     for (size_t x = 0; x < items.size() && (int)x < cap_items; ++x) {

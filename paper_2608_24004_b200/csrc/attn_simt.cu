@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kSimtThreads) attn_simt_kernel(DevPlan P, Attn
 
   for (int it = A.cta_first[blockIdx.x]; it < A.cta_first[blockIdx.x + 1]; ++it) {
     const WorkItem w = A.items[it];
-    const ReqMeta rq = P.req[w.req];
+    const ReqMeta rq{w.n, w.k, w.cu_q, 0};  // (the item's own view of its request: a row block of it, or all of it)
     const int R = G * (rq.k + 1);
     __syncthreads();                        // previous item fully written out before smem is reused
     for (int x = tid; x < R * (D / 8); x += kSimtThreads) {
@@ -161,9 +161,8 @@ template <int DPL>
 __global__ void __launch_bounds__(128) attn_merge_kernel(DevPlan P, AttnArgs A) {
   if ((int)blockIdx.x >= *A.num_merges_dev) return;     // the grid may be sized for the plan's maximum
   const MergeSeg sg = A.merges[blockIdx.x];
-  const ReqMeta rq = P.req[sg.req];
   const int G = P.Hq / P.Hkv;
-  const int R = G * (rq.k + 1);
+  const int R = G * (sg.k + 1);                         // (the pair's own rows: a row block of its request, or all of it)
   const int r = blockIdx.y * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (r >= R) return;
   constexpr int D = DPL * 32;
@@ -190,10 +189,10 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(DevPlan P, AttnArgs A) 
   }
   if (A.sinks) l += exp2f(sk - m);
   const float inv = 1.f / l;
-  __nv_bfloat16* dst = A.out + ((size_t)(rq.cu_q + j) * P.Hq + h) * D + lane * DPL;
+  __nv_bfloat16* dst = A.out + ((size_t)(sg.cu_q + j) * P.Hq + h) * D + lane * DPL;
 #pragma unroll
   for (int c = 0; c < DPL; c += 2) *reinterpret_cast<__nv_bfloat162*>(dst + c) = __floats2bfloat162_rn(o[c] * inv, o[c + 1] * inv);
-  if (A.lse && lane == 0) A.lse[(size_t)(rq.cu_q + j) * P.Hq + h] = (m + log2f(l)) * 0.6931471805599453f;
+  if (A.lse && lane == 0) A.lse[(size_t)(sg.cu_q + j) * P.Hq + h] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
 }  // namespace

@@ -823,7 +823,7 @@ cudaError_t launch_for_rows(int rows, const CUtensorMap& km, const CUtensorMap& 
   if (rows <= 80) return launch_instance<D, 80>(km, vm, P, A, s);
   if (rows <= 96) return launch_instance<D, 96>(km, vm, P, A, s);
   if (rows <= 112) return launch_instance<D, 112>(km, vm, P, A, s);
-  if (rows <= 128) return launch_instance<D, 128>(km, vm, P, A, s);
+  // (wider requests reach this kernel as row blocks of at most 96 rows: see plan_block_positions)
   return cudaErrorInvalidValue;
 }
 
@@ -837,7 +837,8 @@ bool attn_tc_supported(int Hq, int Hkv, int D, int bs, int max_draft, int window
   const int rows = (Hq / Hkv) * (max_draft + 1);
   (void)window;                                       // full attention and sliding windows are both covered
   if (bs != 16 && bs != 32 && bs != 64 && bs != 128) return false;
-  return (D == 128 && rows <= 128) || (D == 64 && rows <= kMaxRows);
+  // (head_dim 128: up to 128 rows per launch item; the planner cuts wider requests into row blocks by draft position)
+  return (D == 128 && rows <= kMaxRows && Hq / Hkv <= kKeysOnMRows) || (D == 64 && rows <= kMaxRows);
 }
 
 int launch_attn_tc(const DevPlan& P, const AttnArgs& A, TcState& st, cudaStream_t s, std::string& err) {

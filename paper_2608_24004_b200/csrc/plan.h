@@ -34,6 +34,7 @@ struct MergeSeg {                     // a pair that was cut into num_parts item
   int32_t kv_head;
   int32_t part_row;                   // partial p of the pair starts at part_row + p * G * (k + 1)
   int32_t num_parts;
+  int32_t k, cu_q;                    // the pair's draft length and first row (a row block's own, see plan_block_positions)
 };
 
 struct KindLayout {                   // byte offsets into the workspace
@@ -72,6 +73,23 @@ __host__ __device__ inline int64_t plan_tile_cost(bool tensor_core, bool rows_on
   const int groups = slabs_inst < 7 ? slabs_inst : 7;                 // softmax warpgroups of the instance
   const int per_group = ((rows + 15) / 16 + groups - 1) / groups;     // 16-row slabs a warpgroup walks per tile
   return 8 + 4 * (per_group - 1);
+}
+
+// Row blocks.  The keys-on-M kernel (head_dim 128) is instantiated for up to 112 query rows per (request, kv-head)
+// pair and is at its best up to 96; a request with more rows is planned as several pairs by rows, of equal size and at
+// most 96 rows where the group size allows: block v covers draft positions [v * pb, (v + 1) * pb), and is to the
+// kernels a request of its own with n' = n + v * pb committed entries (the earlier positions of the same step are in
+// the pages by then: the append precedes the attention), k' = min(k - v * pb, pb - 1) drafts and first row
+// cu_q' = cu_q + v * pb.  Returns pb for a request with k drafts: k + 1 (a single block) when the launch's kernel takes
+// all rows of a pair at once (SIMT, rows on M) or the request has no more than 112.
+constexpr int kKeysOnMRows = 112;     // widest keys-on-M instance
+__host__ __device__ inline int plan_block_positions(bool tensor_core, bool rows_on_m, int G, int k) {
+  const int R = G * (k + 1);
+  if (!tensor_core || rows_on_m || R <= kKeysOnMRows) return k + 1;
+  const int V = (R + 95) / 96;
+  int pb = (k + V) / V;                                  // ceil((k + 1) / V)
+  while (pb > 1 && pb * G > kKeysOnMRows) --pb;          // (one position's G rows always fit: G <= 112 is required)
+  return pb;
 }
 
 // CTA that owns cost unit x when C units are dealt evenly to P CTAs.

@@ -40,6 +40,30 @@ __device__ __forceinline__ int64_t block_scan_excl(int64_t v, int64_t* scratch, 
   return scratch[warp] + incl - v;
 }
 
+// Inclusive prefix maximum of one int per thread over the block (`scratch`: 33 ints).
+__device__ __forceinline__ int block_scan_max_incl(int v, int* scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, v, d);
+    if (lane >= d) v = max(v, up);
+  }
+  __syncthreads();
+  if (lane == 31) scratch[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    int w = lane < (int)(blockDim.x >> 5) ? scratch[lane] : -1;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, w, d);
+      if (lane >= d) w = max(w, up);
+    }
+    scratch[lane] = w;                     // inclusive maximum over warps 0..lane
+  }
+  __syncthreads();
+  return warp > 0 ? max(v, scratch[warp - 1]) : v;
+}
+
 // Leaves an empty step behind (nothing for any later kernel to do) and records why.
 __device__ void write_empty_step(const PlanDevArgs& a) {
   for (int x = threadIdx.x; x < (int)(sizeof(StepHeader) / 4); x += blockDim.x) reinterpret_cast<int32_t*>(a.hdr)[x] = 0;
@@ -51,6 +75,7 @@ __device__ void write_empty_step(const PlanDevArgs& a) {
 __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a) {
   __shared__ int64_t scratch[33];
   __shared__ int s_last_owner[kPlanThreadsMax];
+  __shared__ int s_max[33];
   __shared__ int s_bad;
   const int tid = threadIdx.x;
   const int kPlanThreads = blockDim.x;                 // a multiple of 32, fixed per plan
@@ -112,11 +137,15 @@ __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a)
       int64_t c = 0;
       if (i < B) {
         const ReqMeta r = a.req[i];
-        const int end = r.n + r.k + 1;
-        const int lo = K.window > 0 ? max(0, r.n - K.window + 1) : 0;
-        const int t_count = (end + kTileKeys - 1) / kTileKeys - lo / kTileKeys;
-        const int rows = a.G * (r.k + 1);
-        c = (plan_item_overhead(K.tensor_core, K.rows_on_m, rows) + t_count * plan_tile_cost(K.tensor_core, K.rows_on_m, K.rows_inst, rows)) * a.Hkv;
+        const int pb = plan_block_positions(K.tensor_core, K.rows_on_m, a.G, r.k);
+        for (int first = 0; first <= r.k; first += pb) {                     // the request's row blocks
+          const int n = r.n + first, k = min(r.k - first, pb - 1);
+          const int end = n + k + 1;
+          const int lo = K.window > 0 ? max(0, n - K.window + 1) : 0;
+          const int t_count = (end + kTileKeys - 1) / kTileKeys - lo / kTileKeys;
+          const int rows = a.G * (k + 1);
+          c += (plan_item_overhead(K.tensor_core, K.rows_on_m, rows) + t_count * plan_tile_cost(K.tensor_core, K.rows_on_m, K.rows_inst, rows)) * a.Hkv;
+        }
       }
       int64_t tot;
       block_scan_excl(c, scratch, tot);
@@ -127,8 +156,9 @@ __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a)
       if (tid == 0) a.hdr->num_merges[kd * kMaxSub] = 0;
       continue;
     }
-    // pairs in (request, kv-head) order, 1024 at a time: count the pieces, then emit them
-    const int pairs = B * a.Hkv;
+    // pairs in (request, row block, kv-head) order, 1024 at a time: count the pieces, then emit them.  (A request has one
+    // row block unless the kernel holds fewer rows than it has; blocks beyond its draft length are empty pairs.)
+    const int pairs = B * K.row_blocks * a.Hkv;
     int64_t c0_run = 0;                  // cost units before the chunk's first pair
     int64_t items_run = 0, merges_run = 0, prow_run = 0;
     int last_owner_run = -1;             // owner of the last item emitted so far
@@ -139,17 +169,26 @@ __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a)
       int64_t cpt = 0, pc = 0, ovh = 0;
       ReqMeta r{};
       if (pr < pairs) {
-        i = pr / a.Hkv;
-        g = pr - i * a.Hkv;
+        i = pr / (K.row_blocks * a.Hkv);
+        const int vb = (pr / a.Hkv) % K.row_blocks;
+        g = pr % a.Hkv;
         r = a.req[i];
-        end = r.n + r.k + 1;
-        const int lo = K.window > 0 ? max(0, r.n - K.window + 1) : 0;
-        t_first = lo / kTileKeys;
-        t_count = (end + kTileKeys - 1) / kTileKeys - t_first;
-        R = a.G * (r.k + 1);
-        cpt = plan_tile_cost(K.tensor_core, K.rows_on_m, K.rows_inst, R);
-        ovh = plan_item_overhead(K.tensor_core, K.rows_on_m, R);
-        pc = ovh + t_count * cpt;
+        const int pb = plan_block_positions(K.tensor_core, K.rows_on_m, a.G, r.k);
+        const int first = vb * pb;
+        if (first <= r.k) {
+          // the row block as a request of its own
+          r.n += first;
+          r.k = min(r.k - first, pb - 1);
+          r.cu_q += first;
+          end = r.n + r.k + 1;
+          const int lo = K.window > 0 ? max(0, r.n - K.window + 1) : 0;
+          t_first = lo / kTileKeys;
+          t_count = (end + kTileKeys - 1) / kTileKeys - t_first;
+          R = a.G * (r.k + 1);
+          cpt = plan_tile_cost(K.tensor_core, K.rows_on_m, K.rows_inst, R);
+          ovh = plan_item_overhead(K.tensor_core, K.rows_on_m, R);
+          pc = ovh + t_count * cpt;
+        }
       }
       int64_t chunk_cost;
       const int64_t c0 = c0_run + block_scan_excl(pc, scratch, chunk_cost);
@@ -165,10 +204,11 @@ __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a)
       const int64_t merge0 = merges_run + block_scan_excl(parts > 1 ? 1 : 0, scratch, tm);
       const int64_t prow0 = prow_run + block_scan_excl(parts > 1 ? (int64_t)parts * R : 0, scratch, tp);
       if (items_run + ti > a.max_items || merges_run + tm > a.max_merges || prow_run + tp > a.max_part_rows) overflow = true;
-      s_last_owner[tid] = last_owner;
+      // owner of the last item up to and including this pair (owners never decrease; an empty pair has none of its own)
+      s_last_owner[tid] = max(last_owner_run, block_scan_max_incl(last_owner, s_max));
       __syncthreads();
       if (!overflow && pr < pairs) {
-        // owner of the item before this pair's first: every pair has at least one piece
+        // owner of the item before this pair's first
         const int prev_owner = tid == 0 ? last_owner_run : s_last_owner[tid - 1];
         int po = prev_owner, idx = 0;
         for (int t = 0, t_end, o; t < t_count; t = t_end, ++idx) {
@@ -187,7 +227,7 @@ __global__ void __launch_bounds__(kPlanThreadsMax, 1) plan_kernel(PlanDevArgs a)
           for (int c = po + 1; c <= o; ++c) K.cta_first[c] = (int32_t)(item0 + idx);
           po = o;
         }
-        if (parts > 1) K.merges[merge0] = MergeSeg{i, g, (int32_t)prow0, parts};
+        if (parts > 1) K.merges[merge0] = MergeSeg{i, g, (int32_t)prow0, parts, r.k, r.cu_q};
       }
       const int chunk_last = min(kPlanThreads, pairs - base) - 1;
       const int lo_next = s_last_owner[chunk_last];

@@ -11,6 +11,7 @@ struct PlanDevKind {                  // one layer flavour: where its work list 
   int32_t window;
   int32_t num_ctas;
   int32_t rows_inst;                  // row count the launch is configured for (the plan's maximum)
+  int32_t row_blocks;                 // most row blocks any request can have (plan_block_positions)
   bool tensor_core, rows_on_m;
 };
 

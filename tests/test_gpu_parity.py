@@ -104,6 +104,10 @@ SHAPES = [
     (64, 8, 64, 32, 300, True, [40000, 299, 300, 301], [16, 17, 0, 9]),   # two row blocks under a window, one long split pair
     (8, 8, 64, 16, 0, False, [1000, 129, 0], [16, 1, 0]),            # one query head per kv head: 17, 2 and 1 rows
     (64, 8, 64, 16, 0, True, [500, 3000, 64], [31, 20, 24]),         # 256, 168 and 200 rows: the most head_dim 64 takes
+    (64, 8, 128, 16, 0, True, [1500, 129, 40, 5000], [16, 15, 16, 0]),   # head_dim 128 beyond 128 rows: 136 = two row blocks
+    (64, 8, 128, 16, 0, False, [700, 2600, 127], [23, 17, 31]),      # 192, 144 and 256 rows at head_dim 128
+    (64, 8, 128, 32, 200, True, [40000, 199, 200, 201], [31, 16, 24, 5]),   # row blocks under a window, one long split pair
+    (48, 16, 128, 16, 0, False, [900, 300], [60, 41]),               # three query heads per kv head: blocks of 42 positions
 ]
 
 

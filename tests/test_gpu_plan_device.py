@@ -45,6 +45,9 @@ CASES = [
     (7, 128, 4, 4, 0, 1, 0, "tc", False),           # a single request without drafts
     (8, 128, 32, 8, 0, 300, 3, "tc", False),        # 2400 (request, kv-head) pairs: three chunks of the planner CTA
     (9, 64, 16, 2, 0, 1500, 1, "tc", False),        # 1500 requests: two chunks of requests, three of pairs
+    (10, 128, 64, 8, 0, 7, 16, "tc", False),        # head_dim 128, up to 136 rows: requests cut into two row blocks
+    (11, 128, 32, 4, 150, 5, 31, "tc", True),       # 256 rows: two full row blocks, long contexts, a window
+    (12, 128, 24, 8, 0, 6, 60, "tc", False),        # three query heads per kv head: blocks of 42 positions (126 rows)
 ]
 
 
