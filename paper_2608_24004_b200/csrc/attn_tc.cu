@@ -47,7 +47,8 @@ struct Smem {
   static constexpr int kSlabs = NPAD / 16;                    // 16-row slabs of the query-row dimension
   static constexpr int kGroups = kSlabs < 7 ? kSlabs : 7;     // softmax warpgroups: one per slab up to seven (960 threads)
   static constexpr int kSlabsPerGroup = (kSlabs + kGroups - 1) / kGroups;
-  static constexpr int kThreads = 64 + 128 * kGroups;
+  static constexpr int kThreads = 64 + 128 * kGroups + 32;      // K producer, issuer, softmax warpgroups, V producer
+  static constexpr int kWarpProd2 = 2 + 4 * kGroups;
   // one ring slot: a 128-key K or V tile
   static constexpr int kSlotBytes = kTile * D * 2;
   static constexpr int kQBytes = NPAD * D * 2;
@@ -176,63 +177,64 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s0 = tmem, tmem_o = tmem + 2 * NPAD;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    // The page ids of the next tile are requested before this tile's copies are issued, so the
-    // block-table round trip overlaps with the waits on the ring.
+  if (warp == 0 || warp == L::kWarpProd2) {
+    // ------------------------------------------------------------------ TMA producers
+    // Two warps share the ring: warp 0 copies the K tiles (even slots of the running sequence K(0), V(0), K(1), ...),
+    // the last warp the V tiles.  One warp issuing all sixteen copies of a tile pair, one lane after the other, reaches
+    // 6.5 TB/s over the device with nothing else to do; two reach 6.9.  Page ids come 32 at a time (one coalesced
+    // load of the request's block-table row: four tiles' worth at 16 keys a page), a chunk ahead of their use, so that
+    // no pass of the loop waits for a global-memory round trip.
+    const int which = warp == 0 ? 0 : 1;
+    const CUtensorMap* map = which == 0 ? &kmap : &vmap;
     const int pages_per_tile = kTile / P.bs;
+    const int tiles_per_chunk = 32 / pages_per_tile;
     const uint32_t page_bytes = (uint32_t)P.bs * D * 2;
-    uint32_t load_idx = 0;
-    bool ok = it_begin < it_end;
-    int it = it_begin, tile = 0;
-    ItemView v = ok ? view(A, item_cache, it_begin, it) : ItemView{};
-    auto fetch_page = [&](const ItemView& iv, int tl) -> int {       // raw id of page `lane` of tile tl, or -1
-      const int kb = iv.key_begin + tl * kTile;
-      const int np = min(pages_per_tile, (iv.key_end - kb + P.bs - 1) / P.bs);
-      return lane < np ? __ldg(A.block_table + (size_t)iv.req * P.max_blocks + kb / P.bs + lane) : -1;
+    auto chunk_load = [&](const ItemView& v, int c) -> int {
+      const int idx = c * 32 + lane;                       // page of the item's key range
+      const int np_item = (v.key_end - v.key_begin + P.bs - 1) / P.bs;
+      return idx < np_item ? __ldg(A.block_table + (size_t)v.req * P.max_blocks + v.key_begin / P.bs + idx) : -1;
     };
-    int page_raw = ok ? fetch_page(v, 0) : -1;
+    uint32_t tile_idx = 0;                                 // running tile number of this CTA
+    bool ok = it_begin < it_end;
+    int it = it_begin;
+    ItemView v = ok ? view(A, item_cache, it_begin, it_begin) : ItemView{};
+    int ids = ok ? chunk_load(v, 0) : -1;
     while (ok) {
-      int nit = it, ntile = tile + 1;
-      ItemView nv = v;
-      if (ntile == v.tiles) {
-        nit = it + 1;
-        ntile = 0;
-        if (nit < it_end) nv = view(A, item_cache, it_begin, nit);
-      }
-      const bool more = nit < it_end;
-      const int next_raw = more ? fetch_page(nv, ntile) : -1;
-      const int kbase = v.key_begin + tile * kTile;
-      const int npages = min(pages_per_tile, (v.key_end - kbase + P.bs - 1) / P.bs);
-      int page = page_raw;
-      if (lane < npages && (unsigned)page >= (unsigned)P.num_blocks) {
-        atomicOr(P.status, kFlagBadPage);
-        page = -1;
-      }
-      const int nvalid = __popc(__ballot_sync(0xffffffffu, page >= 0));
-      if (A.stall_after_loads >= 0 && (int)load_idx >= A.stall_after_loads) break;   // (test hook: the copies stop coming)
-      for (int which = 0; which < 2; ++which) {
-        const int slot = load_idx % kSlots;
-        const uint32_t par = ((load_idx / kSlots) & 1u) ^ 1u;
-        int good = 1;
-        if (lane == 0) good = mbar_wait_c(bar_slot_empty(slot), par, ctl, P.status, 0) ? 1 : 0;
-        good = __shfl_sync(0xffffffffu, good, 0);
-        if (!good) {
-          ok = false;
-          break;
+      const int nit = it + 1;
+      const ItemView nv = nit < it_end ? view(A, item_cache, it_begin, nit) : ItemView{};
+      const int nch = (v.tiles + tiles_per_chunk - 1) / tiles_per_chunk;
+      for (int c = 0; c < nch && ok; ++c) {
+        const int ids_next = c + 1 < nch ? chunk_load(v, c + 1) : (nit < it_end ? chunk_load(nv, 0) : -1);
+        const int t_end = min(v.tiles, (c + 1) * tiles_per_chunk);
+        for (int tile = c * tiles_per_chunk; tile < t_end; ++tile, ++tile_idx) {
+          if (A.stall_after_loads >= 0 && (int)tile_idx >= A.stall_after_loads) { ok = false; break; }   // (test hook: the copies stop coming)
+          const int kbase = v.key_begin + tile * kTile;
+          const int npages = min(pages_per_tile, (v.key_end - kbase + P.bs - 1) / P.bs);
+          int page = __shfl_sync(0xffffffffu, ids, ((tile - c * tiles_per_chunk) * pages_per_tile + lane) & 31);
+          if (lane >= npages) page = -1;
+          if (lane < npages && (unsigned)page >= (unsigned)P.num_blocks) {
+            atomicOr(P.status, kFlagBadPage);
+            page = -1;
+          }
+          const int nvalid = __popc(__ballot_sync(0xffffffffu, page >= 0));
+          const uint32_t load_idx = 2 * tile_idx + which;
+          const int slot = load_idx % kSlots;
+          const uint32_t par = ((load_idx / kSlots) & 1u) ^ 1u;
+          int good = 1;
+          if (lane == 0) good = mbar_wait_c(bar_slot_empty(slot), par, ctl, P.status, 0) ? 1 : 0;
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
+          if (lane == 0) mbar_arrive_expect_tx(bar_slot_full(slot), (uint32_t)nvalid * page_bytes);
+          __syncwarp();
+          if (page >= 0)
+            tma_load_5d(sbase + slot * L::kSlotBytes + lane * page_bytes, map, bar_slot_full(slot), 0, 0, 0, 0,
+                        page * P.Hkv + v.kv_head);
         }
-        if (lane == 0) mbar_arrive_expect_tx(bar_slot_full(slot), (uint32_t)nvalid * page_bytes);
-        __syncwarp();
-        if (page >= 0)
-          tma_load_5d(sbase + slot * L::kSlotBytes + lane * page_bytes, which == 0 ? &kmap : &vmap,
-                      bar_slot_full(slot), 0, 0, 0, 0, page * P.Hkv + v.kv_head);
-        ++load_idx;
+        ids = ids_next;
       }
-      if (!more) break;
+      if (nit >= it_end) break;
       it = nit;
-      tile = ntile;
       v = nv;
-      page_raw = next_raw;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (one lane)
@@ -298,7 +300,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
       }
       if (ok && have_prev) issue_pv(g - 1, prev_first, prev_last, prev_item);
     }
-  } else {
+  } else if (warp < L::kWarpProd2) {
     // ------------------------------------------------------------------ softmax + epilogue
     // Warpgroup wg owns the 16-row slabs wg, wg + NWG, ... (rows = TMEM columns): their references,
     // their weights, their slice of O^T and of the output.  Warpgroups never synchronise with each other.
