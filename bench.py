@@ -148,6 +148,44 @@ def other_workload(bnd, label, b, dev, steps, target_ms=250.0):
         attn_ms = statistics.mean(row[kind][0].elapsed_time(row[kind][1]) for row in pairs)
         entry["layers"].append({"kind": kind, "window": int(b.kinds[kind].window), "roofline": roofline_of(bnd, b, vs, kind, attn_ms)})
     entry["roofline"] = entry["layers"][-1]["roofline"]
+    if b.temperature is not None:
+        # the same step with the hidden states as the acceptance input (as_accept_lm_head_sampled): the [rows, vocab]
+        # logits and what reads them are replaced by the projection itself, two passes over the weights (every row for
+        # the accept test, then one row per request for the recovery draw).  Seeded random hidden states and weights:
+        # the drafts of this workload were drawn from its own logits, so nearly every request rejects its first draft
+        # here; the work of the call does not depend on that.
+        H = HIDDEN_DIM.get(b.name, 4096) // 64 * 64
+        g = torch.Generator(device="cuda").manual_seed(78)
+        hidden = torch.randn((b.total_q, H), generator=g, device="cuda").to(torch.bfloat16)
+        weight = torch.empty((b.vocab, H), dtype=torch.bfloat16, device="cuda")
+        for at in range(0, b.vocab, 16384):
+            weight[at:at + 16384] = (torch.randn((min(16384, b.vocab - at), H), generator=g, device="cuda") * (2.0 / H ** 0.5)).to(torch.bfloat16)
+        scratch = torch.empty(bnd.as_accept_lm_head_scratch_bytes(vs.plan, H, b.vocab), dtype=torch.uint8, device="cuda")
+        acc_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(10)]
+
+        def run_lm(n, ev=None):
+            for i in range(n):
+                vs.block_table.copy_(bt0); vs.seq_lens.copy_(seq0)
+                vs.plan_step()
+                for kind in range(n_kinds):
+                    vs.attn(kind)
+                if ev is not None:
+                    ev[i][0].record()
+                bnd.as_accept_lm_head_sampled(vs.plan, hidden, weight, vs.draft_tokens, vs.draft_probs, vs.temperature, vs.u, vs.w,
+                                              None, scratch, vs.accept_len, vs.out_tokens)
+                if ev is not None:
+                    ev[i][1].record()
+                vs.commit(kind=n_kinds - 1)
+        run_lm(3)
+        e0.record(); run_lm(10, acc_ev); e1.record()
+        torch.cuda.synchronize()
+        assert bnd.as_plan_check(vs.plan) == 0
+        acc_ms = statistics.mean(a.elapsed_time(c) for a, c in acc_ev)
+        flops = 2.0 * (b.total_q + b.batch) * H * b.vocab
+        entry["from_hidden_states"] = {"ms_per_step": e0.elapsed_time(e1) / 10, "accept_call_ms": acc_ms, "rows": b.total_q,
+                                       "recovery_rows": b.batch, "hidden_dim": H, "vocab": b.vocab,
+                                       "tflops": flops / (acc_ms * 1e-3) / 1e12,
+                                       "logits_bytes_not_materialised": b.total_q * b.vocab * 4}
     return entry
 
 

@@ -211,6 +211,26 @@ AS_API int as_accept_seeded(as_plan_t* plan, const float* logits, int64_t ld, in
 AS_API int as_accept_lm_head(as_plan_t* plan, const void* hidden, const void* weight, int hidden_dim, int vocab,
                       const int32_t* draft_tokens, int32_t* accept_len, int32_t* out_tokens, void* stream);
 
+/* The same fusion for sampling requests (lossless rejection sampling, the reading of as_accept): the projection
+ * is computed tile by tile and reduced at once to what the accept test needs of a row - its argmax, the online pair
+ * (max, sum of exp((z - max) / T)) and the single logit z[d] of the row's draft token - so that p[d] is known without
+ * any logits in memory; the extra token is then drawn from the recovery distribution of ONE row per request (row a_i),
+ * whose logits a second, small pass over the weights writes to `scratch` (batch rows instead of total_q).
+ *   hidden, weight, hidden_dim, vocab, draft_tokens, accept_len, out_tokens: as for as_accept_lm_head.
+ *   draft_probs: dev fp32 [total_d, ld] (ld >= vocab) or NULL for a one-hot drafter; temperature: dev fp32 [batch],
+ *     required (T_i <= 0 = greedy for that request); u, w: dev fp32 [total_d], [total_q]; or rng_state: dev uint64 [2]
+ *     {seed, step} for uniforms drawn in the kernels exactly as as_accept_seeded draws them (then u, w may be NULL).
+ *   scratch: dev, 256-byte aligned, at least as_accept_lm_head_scratch_bytes(plan, hidden_dim, vocab) bytes (sized
+ *     for the plan's maxima); contents are scratch.
+ * Decisions equal as_accept's on the logits hidden x weight^T except where a ratio min(1, p/q) lies within the
+ * projection's accumulation error of its uniform (the tensor cores sum bf16 products in fp32, in their own order). */
+AS_API size_t as_accept_lm_head_scratch_bytes(const as_plan_t* plan, int hidden_dim, int vocab);
+AS_API int as_accept_lm_head_sampled(as_plan_t* plan, const void* hidden, const void* weight, int hidden_dim, int vocab,
+                                     const int32_t* draft_tokens, const float* draft_probs, int64_t ld,
+                                     const float* temperature, const float* u, const float* w, const uint64_t* rng_state,
+                                     void* scratch, size_t scratch_bytes, int32_t* accept_len, int32_t* out_tokens,
+                                     void* stream);
+
 /* Commit / rollback (paper: silent; this is the bookkeeping any paged cache needs after a verify
  * step).  seq_lens: dev int32 [batch], in: n_i, out: n_i + a_i + 1.  Every page of request i with
  * logical index >= ceil(n_i'/bs) that the step held is released: its table entry becomes -1 and

@@ -23,7 +23,7 @@ AS_COMMIT_SCRUB = 1
 AS_ATTN_AUTO, AS_ATTN_SIMT, AS_ATTN_TC = 0, 1, 2
 
 EXPORTS = ["as_status_string", "as_last_error", "as_plan_create", "as_plan_destroy", "as_plan_workspace_bytes",
-           "as_plan_bind", "as_plan_set_attn_impl", "as_plan_set_fixed_launch", "as_plan", "as_plan_device", "as_verify_attn", "as_accept", "as_accept_seeded", "as_accept_lm_head", "as_kv_commit",
+           "as_plan_bind", "as_plan_set_attn_impl", "as_plan_set_fixed_launch", "as_plan", "as_plan_device", "as_verify_attn", "as_accept", "as_accept_seeded", "as_accept_lm_head", "as_accept_lm_head_sampled", "as_accept_lm_head_scratch_bytes", "as_kv_commit",
            "as_plan_check", "as_plan_stats", "as_plan_preview", "as_plan_set_profile_events", "as_plan_launch_count", "as_plan_set_test_stall", "as_budget",
            "as_accept_greedy_static", "as_drafter_create", "as_drafter_destroy", "as_drafter_open", "as_drafter_close", "as_drafter_forget",
            "as_drafter_feed", "as_drafter_block", "as_drafter_propose"]
@@ -63,6 +63,10 @@ def _load():
     lib.as_plan_launch_count.argtypes = [C.c_void_p]
     lib.as_plan_launch_count.restype = C.c_int64
     lib.as_plan_set_test_stall.argtypes = [C.c_void_p, C.c_uint64, C.c_int]
+    lib.as_accept_lm_head_scratch_bytes.restype = C.c_size_t
+    lib.as_accept_lm_head_scratch_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
+    lib.as_accept_lm_head_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64] \
+        + [C.c_void_p] * 5 + [C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.as_budget.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_double, C.c_double, C.c_int, C.c_void_p,
                               C.c_void_p]
     lib.as_accept_greedy_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
@@ -189,6 +193,26 @@ def as_accept_lm_head(plan: Plan, hidden: torch.Tensor, weight: torch.Tensor, dr
     _chk(_lib.as_accept_lm_head(plan.handle, _dptr(hidden, bf), _dptr(weight, bf), hidden.shape[1], weight.shape[0],
                                 _dptr(draft_tokens, i32, True), _dptr(accept_len, i32), _dptr(out_tokens, i32),
                                 _stream(stream)), "as_accept_lm_head")
+
+
+def as_accept_lm_head_scratch_bytes(plan: Plan, hidden_dim: int, vocab: int) -> int:
+    return int(_lib.as_accept_lm_head_scratch_bytes(plan.handle, hidden_dim, vocab))
+
+
+def as_accept_lm_head_sampled(plan: Plan, hidden: torch.Tensor, weight: torch.Tensor, draft_tokens, draft_probs, temperature,
+                              u, w, rng_state, scratch: torch.Tensor, accept_len, out_tokens, stream=None):
+    """Rejection sampling from hidden states [rows, H] and the output projection's weights [V, H] (both bf16); scratch is a
+    uint8 tensor of at least as_accept_lm_head_scratch_bytes() bytes; u / w or rng_state (uint64 {seed, step}) as in as_accept."""
+    bf, i32, f32 = torch.bfloat16, torch.int32, torch.float32
+    assert hidden.dim() == 2 and weight.dim() == 2 and hidden.shape[1] == weight.shape[1]
+    assert draft_probs is None or (draft_probs.dim() == 2 and draft_probs.stride(1) == 1)
+    _chk(_lib.as_accept_lm_head_sampled(plan.handle, _dptr(hidden, bf), _dptr(weight, bf), hidden.shape[1], weight.shape[0],
+                                        _dptr(draft_tokens, i32, True), _dptr(draft_probs, f32, True),
+                                        0 if draft_probs is None else draft_probs.stride(0), _dptr(temperature, f32),
+                                        _dptr(u, f32, True), _dptr(w, f32, True),
+                                        None if rng_state is None else C.c_void_p(rng_state.data_ptr()),
+                                        C.c_void_p(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
+                                        _dptr(accept_len, i32), _dptr(out_tokens, i32), _stream(stream)), "as_accept_lm_head_sampled")
 
 
 def as_plan_device(plan: Plan, batch: int, seq_lens: torch.Tensor, draft_lens: torch.Tensor, block_table: torch.Tensor,

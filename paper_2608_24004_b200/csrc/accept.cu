@@ -216,7 +216,7 @@ __global__ void decide_kernel(DevPlan P, AcceptArgs A) {
       } else if (!sampling) {
         ok = (__float_as_int(rf.y) == d);
       } else {
-        const float zd = clean(A.logits[(size_t)(rq.cu_q + j) * A.ld + d]);
+        const float zd = clean(A.zd ? A.zd[rq.cu_q + j] : A.logits[(size_t)(rq.cu_q + j) * A.ld + d]);
         const float pd = exp2f(zd * (kLog2e / T) - rf.z) / rf.w;
         const float qd = A.draft_probs ? A.draft_probs[(size_t)(rq.cu_d + j) * A.ld + d] : 1.f;
         float ratio;
@@ -258,7 +258,7 @@ __device__ __forceinline__ RecRow rec_row(const DevPlan& P, const AcceptArgs& A,
   const ReqMeta rq = P.req[i];
   RecRow r;
   const int row = rq.cu_q + a;
-  r.z = A.logits + (size_t)row * A.ld;
+  r.z = A.rec_logits ? A.rec_logits + (size_t)i * A.rec_ld : A.logits + (size_t)row * A.ld;
   r.bonus = (a == rq.k);
   r.q = (!r.bonus && A.draft_probs) ? A.draft_probs + (size_t)(rq.cu_d + a) * A.ld : nullptr;
   r.onehot = (!r.bonus && !A.draft_probs) ? A.draft_tokens[rq.cu_d + a] : -1;
@@ -498,6 +498,18 @@ cudaError_t launch_accept(const DevPlan& P, const AcceptArgs& A, cudaStream_t s)
     e = cudaGetLastError();
   }
   return e;
+}
+
+cudaError_t launch_recover(const DevPlan& P, const AcceptArgs& A, cudaStream_t s) {
+  if (P.batch == 0) return cudaSuccess;
+  recover_den_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  recover_cells_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  recover_pick_kernel<<<(P.batch + 3) / 4, 128, 0, s>>>(P, A);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_decide(const DevPlan& P, const AcceptArgs& A, cudaStream_t s) {

@@ -93,6 +93,7 @@ struct as_plan_s {
   std::vector<char> host_meta;
   TcState tc;                 // tensor-map cache of the tensor-core kernel
   LmHeadState lm;             // tensor-map cache of the fused output projection
+  LmHeadState lm_rec;         // ... of its second pass over the recovery rows (as_accept_lm_head_sampled)
   cudaEvent_t prof_begin = nullptr, prof_end = nullptr;
   unsigned long long test_wait_limit_ns = 0;   // as_plan_set_test_stall
   int test_stall_after_loads = -1;
@@ -775,6 +776,88 @@ int as_accept_lm_head(as_plan_t* p, const void* hidden, const void* weight, int 
   if (rc != 0) return fail(rc, "as_accept_lm_head: " + err);
   AS_CUDA(launch_decide(d, A, s));
   p->launches += 3;
+  return AS_OK;
+}
+
+size_t as_accept_lm_head_scratch_bytes(const as_plan_t* p, int hidden_dim, int vocab) {
+  if (!p || hidden_dim < 1 || vocab < 1) return 0;
+  const size_t ld = align_up((size_t)vocab, 4);
+  const size_t logits = sizeof(float) * (size_t)p->max_batch * ld;
+  const size_t parts = sizeof(float2) * (size_t)p->max_total_q * lm_head_vocab_tiles(vocab);
+  return align_up(std::max(logits, parts), 256) + align_up(sizeof(uint16_t) * (size_t)p->max_batch * hidden_dim, 256) +
+         align_up(sizeof(float) * (size_t)p->max_total_q, 256);
+}
+
+int as_accept_lm_head_sampled(as_plan_t* p, const void* hidden, const void* weight, int hidden_dim, int vocab,
+                              const int32_t* draft_tokens, const float* draft_probs, int64_t ld, const float* temperature,
+                              const float* u, const float* w, const uint64_t* rng_state, void* scratch, size_t scratch_bytes,
+                              int32_t* accept_len, int32_t* out_tokens, void* stream) {
+  if (!p || !hidden || !weight || !accept_len || !out_tokens || !temperature || !scratch)
+    return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: null pointer");
+  if (!p->planned) return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: as_plan() has not been called for this step");
+  if (vocab < 1 || hidden_dim < 64 || hidden_dim % 64 != 0)
+    return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: need vocab >= 1 and hidden_dim a positive multiple of 64");
+  if (!rng_state && (!u || !w)) return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: sampling needs u and w, or rng_state");
+  if (draft_probs && ld < vocab) return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: need ld >= vocab for draft_probs");
+  if ((reinterpret_cast<uintptr_t>(hidden) | reinterpret_cast<uintptr_t>(weight)) & 15)
+    return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: hidden and weight must be 16-byte aligned");
+  if ((reinterpret_cast<uintptr_t>(scratch) & 255) || scratch_bytes < as_accept_lm_head_scratch_bytes(p, hidden_dim, vocab))
+    return fail(AS_ERR_WORKSPACE, "as_accept_lm_head_sampled: scratch not 256-byte aligned or smaller than as_accept_lm_head_scratch_bytes()");
+  if (p->total_d > 0 && !draft_tokens) return fail(AS_ERR_INVALID_ARG, "as_accept_lm_head_sampled: draft_tokens is null");
+  if (p->batch == 0) return AS_OK;
+  DeviceGuard guard(p->device);
+  if (!guard.ok) return fail(AS_ERR_CUDA, "as_accept_lm_head_sampled: cannot select the plan's device");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const DevPlan d = dev_plan(p);
+  // scratch: [logits of the recovery rows | tile partials of the first pass (dead before the logits are written)]
+  // [hidden states of the recovery rows] [logit of every row's draft token]
+  const size_t rec_ld = align_up((size_t)vocab, 4);
+  char* sc = static_cast<char*>(scratch);
+  const size_t logits_bytes = sizeof(float) * (size_t)p->max_batch * rec_ld;
+  const size_t parts_bytes = sizeof(float2) * (size_t)p->max_total_q * lm_head_vocab_tiles(vocab);
+  float* rec_logits = reinterpret_cast<float*>(sc);
+  float2* tile_part = reinterpret_cast<float2*>(sc);
+  char* hidden_rows = sc + align_up(std::max(logits_bytes, parts_bytes), 256);
+  float* zd = reinterpret_cast<float*>(hidden_rows + align_up(sizeof(uint16_t) * (size_t)p->max_batch * hidden_dim, 256));
+  AcceptArgs A{};
+  A.ld = draft_probs ? ld : vocab;
+  A.vocab = vocab;
+  A.draft_tokens = draft_tokens;
+  A.draft_probs = draft_probs;
+  A.temperature = temperature;
+  A.u = u;
+  A.w = w;
+  A.rng = rng_state;
+  A.accept_len = accept_len;
+  A.out_tokens = out_tokens;
+  A.row_final = reinterpret_cast<float4*>(p->ws + p->off_row_final);
+  A.recover_row = reinterpret_cast<int32_t*>(p->ws + p->off_recover);
+  A.rec_den = reinterpret_cast<double*>(p->ws + p->off_rec_den);
+  A.rec_cells = reinterpret_cast<double*>(p->ws + p->off_rec_cells);
+  A.zd = zd;
+  A.rec_logits = rec_logits;
+  A.rec_ld = (int64_t)rec_ld;
+  int chunk = 16384;
+  while ((vocab + chunk - 1) / chunk > p->accept_chunks_max) chunk *= 2;
+  A.chunk_elems = chunk;
+  A.chunks = (vocab + chunk - 1) / chunk;
+  int cell = 128;
+  while ((vocab + cell - 1) / cell > p->accept_cells_max) cell *= 2;
+  A.cell_elems = cell;
+  A.cells = (vocab + cell - 1) / cell;
+  std::string err;
+  // pass 1 over the weights: argmax, softmax statistics per row, the logit of each draft token
+  int rc = launch_lm_head_stats(d, p->lm, hidden, weight, hidden_dim, vocab, d.total_q, p->num_sms,
+                                reinterpret_cast<unsigned long long*>(p->ws + p->off_row_part), tile_part, zd, draft_tokens,
+                                temperature, A.row_final, s, err);
+  if (rc != 0) return fail(rc, "as_accept_lm_head_sampled: " + err);
+  AS_CUDA(launch_decide(d, A, s));
+  // pass 2, over the one row per request whose recovery distribution is sampled
+  rc = launch_lm_head_recover_rows(d, p->lm_rec, A.recover_row, hidden, hidden_rows, weight, hidden_dim, vocab, d.batch, p->num_sms,
+                                   rec_logits, (long long)rec_ld, s, err);
+  if (rc != 0) return fail(rc, "as_accept_lm_head_sampled: " + err);
+  AS_CUDA(launch_recover(d, A, s));
+  p->launches += 9;
   return AS_OK;
 }
 

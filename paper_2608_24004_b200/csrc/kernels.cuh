@@ -43,6 +43,11 @@ struct AcceptArgs {
   const float* u;
   const float* w;
   const uint64_t* rng;        // device {seed, step}: when set, u and w are drawn in the kernels instead (Philox4x32-10)
+  // acceptance from hidden states: no [total_q, ld] logits exist.  zd [total_q] holds the logit of each row's draft
+  // token, rec_logits [batch, rec_ld] the logits of the one row per request that recovery samples (row a_i)
+  const float* zd = nullptr;
+  const float* rec_logits = nullptr;
+  int64_t rec_ld = 0;
   int32_t* accept_len;
   int32_t* out_tokens;
   // scratch in the workspace

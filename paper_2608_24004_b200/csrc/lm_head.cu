@@ -9,6 +9,11 @@
 // of the next.  Warp 0 issues the TMA copies, one lane of warp 1 the tcgen05.mma, warps 2..5 reduce (thread = row
 // = TMEM lane).  Units (vocabulary tile, row tile) are dealt round-robin with the row tile fastest, so the CTAs
 // that share a weight tile read it at the same time and all but the first find it in L2.  Every wait is bounded.
+//
+// Three epilogues share the pipeline (template parameter): the row argmax alone (greedy acceptance); the argmax plus
+// what rejection sampling needs of a row - per vocabulary tile the online pair (max, sum of 2^((z - max) / T)) and the
+// logit of the row's draft token - for as_accept_lm_head_sampled; and plain fp32 logits stored to memory, which that
+// call uses for the one row per request whose recovery distribution has to be sampled.
 #include <cuda.h>
 
 #include "lm_head.cuh"
@@ -37,9 +42,22 @@ __device__ __forceinline__ unsigned long long pack_key(float v, int col) {
   return ((unsigned long long)ord << 32) | (0xffffffffu - (uint32_t)col);
 }
 
+constexpr int kEpiArgmax = 0, kEpiStats = 1, kEpiStore = 2;
+struct LmEpilogue {
+  unsigned long long* keys;         // argmax, stats: packed (largest logit, its column) per row, folded with atomicMax
+  float2* tile_part;                // stats: [rows, n_tiles] (max, sum) of 2^(z log2e / T - max) over the tile, log2 units
+  float* zd;                        // stats: [rows] logit of the row's draft token
+  const int32_t* draft_tokens;      // stats
+  const float* temperature;         // stats: per request; <= 0 = greedy (no statistics)
+  float* store;                     // store: [rows, store_ld] fp32 logits
+  long long store_ld;
+  int rows;                         // rows of the A operand that exist (the step's rows, or the batch for the store pass)
+};
+
+template <int EPI>
 __global__ void __launch_bounds__(kLmThreads, 1)
-lm_head_argmax_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap wmap, DevPlan P,
-                      int H, int V, int m_tiles, int n_tiles, unsigned long long* __restrict__ keys) {
+lm_head_kernel(const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap wmap, DevPlan P,
+               int H, int V, int m_tiles, int n_tiles, LmEpilogue E) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -50,7 +68,7 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap amap, const __grid_con
   auto bar_acc_free = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); };
   Ctl* ctl = reinterpret_cast<Ctl*>(smem + kStages * kStageBytes + 16 * 8);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int total_q = P.hdr->total_q;
+  const int total_q = EPI == kEpiStore ? min(E.rows, P.hdr->batch) : P.hdr->total_q;
   const int units = m_tiles * n_tiles;
   const int KB = H / kBK;
   constexpr uint32_t TMEM_COLS = 512;
@@ -137,28 +155,96 @@ lm_head_argmax_kernel(const __grid_constant__ CUtensorMap amap, const __grid_con
       if (!mbar_wait(bar_acc_full(buf), (ul >> 1) & 1u, ctl, P.status, 3)) break;
       tc_fence_after();
       const int col0 = n * kBN;
-      float best = -INFINITY;                             // NaN never compares greater: it counts as -inf
-      int best_col = col0;
+      const int r = m * kBM + row;
+      if constexpr (EPI == kEpiStore) {
+        // the tile's logits as they are, 128 bytes per thread and chunk
+        float* dst = E.store + (size_t)r * E.store_ld + col0;
 #pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        float y[32];
-        tmem_ld32(tmem + buf * kBN + lane_addr + c * 32, y);
-        tmem_wait_ld();
+        for (int c = 0; c < kBN / 32; ++c) {
+          float y[32];
+          tmem_ld32(tmem + buf * kBN + lane_addr + c * 32, y);
+          tmem_wait_ld();
+          if (r < total_q) {
+            if (col0 + c * 32 + 31 < V && (E.store_ld & 3) == 0) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float v = y[e] + 0.f;                     // -0 becomes +0: equal logits must tie
-          const int col = col0 + c * 32 + e;
-          if (col < V && v > best) {                      // strict: the lowest column of a tie stays
-            best = v;
-            best_col = col;
+              for (int e = 0; e < 32; e += 4) *reinterpret_cast<float4*>(dst + c * 32 + e) = make_float4(y[e], y[e + 1], y[e + 2], y[e + 3]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (col0 + c * 32 + e < V) dst[c * 32 + e] = y[e];
+            }
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_free(buf));
+      } else {
+        float best = -INFINITY;                             // NaN never compares greater: it counts as -inf
+        int best_col = col0;
+        // what a sampling request's row needs besides: scale of its exponent, its draft token, running (max, sum)
+        float cT = 0.f, sm = -INFINITY, ss = 0.f;
+        int d = -1;
+        if constexpr (EPI == kEpiStats) {
+          if (r < total_q) {
+            const int2 rj = P.row_map[r];
+            const float T = E.temperature[rj.x];
+            if (T > 0.f) {
+              cT = 1.4426950408889634f / T;
+              const ReqMeta rq = P.req[rj.x];
+              if (rj.y < rq.k) d = E.draft_tokens[rq.cu_d + rj.y];
+            }
+          }
+        }
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          float y[32];
+          tmem_ld32(tmem + buf * kBN + lane_addr + c * 32, y);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float v = y[e] + 0.f;                     // -0 becomes +0: equal logits must tie
+            const int col = col0 + c * 32 + e;
+            if (col < V && v > best) {                      // strict: the lowest column of a tie stays
+              best = v;
+              best_col = col;
+            }
+          }
+          if constexpr (EPI == kEpiStats) {
+            if (cT > 0.f) {
+              // entries past the vocabulary (zero fill of the copy) and NaN count as -inf
+              float mx = -INFINITY;
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                if (col0 + c * 32 + e >= V || y[e] != y[e]) y[e] = -INFINITY;
+                mx = fmaxf(mx, y[e]);
+              }
+              const float mnew = fmaxf(sm, mx * cT);
+              if (mnew > -INFINITY) {
+                float add = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) add += exp2f(fmaf(y[e], cT, -mnew));
+                ss = ss * exp2f(sm - mnew) + add;           // sm = -inf: ss is 0 and 2^-inf = 0
+                sm = mnew;
+              }
+              const int de = d - (col0 + c * 32);
+              if (de >= 0 && de < 32) {
+                float zd = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (e == de) zd = y[e];
+                E.zd[r] = zd;
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_free(buf));
+        if (r < total_q) {
+          atomicMax(E.keys + r, pack_key(best, best_col));
+          if constexpr (EPI == kEpiStats) E.tile_part[(size_t)r * n_tiles + n] = make_float2(sm, ss);
+        }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_acc_free(buf));
-      const int r = m * kBM + row;
-      if (r < total_q) atomicMax(keys + r, pack_key(best, best_col));
       ++ul;
     }
   }
@@ -186,6 +272,49 @@ __global__ void lm_head_finish_kernel(DevPlan P, const unsigned long long* __res
   row_final[r] = make_float4(__uint_as_float(bits), __int_as_float(col), 0.f, 0.f);
 }
 
+// The same for a sampling step: the tile partials of a row folded in tile order by one warp (fixed order: the result
+// does not depend on which CTA computed which tile) into (scaled max, sum) beside the argmax.
+__global__ void lm_head_finish_stats_kernel(DevPlan P, const unsigned long long* __restrict__ keys,
+                                            const float2* __restrict__ tile_part, int n_tiles, float4* __restrict__ row_final) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= P.hdr->total_q) return;
+  float m = -INFINITY, s = 0.f;
+  for (int t = lane; t < n_tiles; t += 32) {
+    const float2 p = tile_part[(size_t)r * n_tiles + t];
+    if (p.x == -INFINITY) continue;
+    const float mm = fmaxf(m, p.x);
+    s = (m == -INFINITY ? 0.f : s * exp2f(m - mm)) + p.y * exp2f(p.x - mm);
+    m = mm;
+  }
+  for (int o = 16; o; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    if (m2 != -INFINITY) {
+      const float mm = fmaxf(m, m2);
+      s = (m == -INFINITY ? 0.f : s * exp2f(m - mm)) + s2 * exp2f(m2 - mm);
+      m = mm;
+    }
+  }
+  if (lane == 0) {
+    const unsigned long long k = keys[r];
+    const uint32_t ord = (uint32_t)(k >> 32);
+    const uint32_t bits = ord ^ ((ord >> 31) ? 0x80000000u : 0xffffffffu);
+    const int col = (int)(0xffffffffu - (uint32_t)k);
+    row_final[r] = make_float4(__uint_as_float(bits), __int_as_float(col), m, s);
+  }
+}
+
+// hidden state of the row each sampling request draws its extra token from (row a_i), gathered into [batch, H];
+// zeros for requests that do not sample
+__global__ void lm_head_gather_rows_kernel(DevPlan P, const int32_t* __restrict__ recover_row, const uint4* __restrict__ hidden,
+                                           uint4* __restrict__ out, int H8) {
+  const int i = blockIdx.x;
+  if (i >= P.hdr->batch) return;
+  const int a = recover_row[i];
+  const uint4* src = a >= 0 ? hidden + (size_t)(P.req[i].cu_q + a) * H8 : nullptr;
+  for (int x = threadIdx.x; x < H8; x += blockDim.x) out[(size_t)i * H8 + x] = src ? src[x] : make_uint4(0, 0, 0, 0);
+}
+
 bool encode_2d(void* map, const void* base, uint64_t inner, uint64_t rows, uint32_t box_rows, std::string& err) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) {
@@ -208,38 +337,101 @@ bool encode_2d(void* map, const void* base, uint64_t inner, uint64_t rows, uint3
 
 }  // namespace
 
-int launch_lm_head_argmax(const DevPlan& P, LmHeadState& st, const void* hidden, const void* weight, int H, int V, int rows_extent,
-                          int num_sms, unsigned long long* keys, float4* row_final, cudaStream_t s, std::string& err) {
-  if (rows_extent <= 0) return 0;
+namespace {
+
+bool refresh_maps(LmHeadState& st, const void* hidden, const void* weight, int H, int V, int rows_extent, std::string& err) {
   if (st.hidden != hidden || st.weight != weight || st.H != H || st.V != V || st.rows != rows_extent) {
-    if (!encode_2d(st.a_map, hidden, (uint64_t)H, (uint64_t)rows_extent, kBM, err)) return 4;
-    if (!encode_2d(st.w_map, weight, (uint64_t)H, (uint64_t)V, kBN, err)) return 4;
+    if (!encode_2d(st.a_map, hidden, (uint64_t)H, (uint64_t)rows_extent, kBM, err)) return false;
+    if (!encode_2d(st.w_map, weight, (uint64_t)H, (uint64_t)V, kBN, err)) return false;
     st.hidden = hidden;
     st.weight = weight;
     st.H = H;
     st.V = V;
     st.rows = rows_extent;
   }
+  return true;
+}
+
+template <int EPI>
+cudaError_t launch_epilogue(const LmHeadState& st, const DevPlan& P, int H, int V, int rows_extent, int num_sms, const LmEpilogue& E,
+                            cudaStream_t s) {
   static bool opted_in[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess && (dev < 0 || dev >= 64 || !opted_in[dev])) {
-    e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmem);
+    e = cudaFuncSetAttribute(lm_head_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLmSmem);
     if (e == cudaSuccess && dev >= 0 && dev < 64) opted_in[dev] = true;
   }
-  if (e == cudaSuccess) e = cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)rows_extent, s);
-  if (e == cudaSuccess) {
-    const int m_tiles = (rows_extent + kBM - 1) / kBM, n_tiles = (V + kBN - 1) / kBN;
-    const int grid = m_tiles * n_tiles < num_sms ? m_tiles * n_tiles : num_sms;
-    lm_head_argmax_kernel<<<grid, kLmThreads, kLmSmem, s>>>(*reinterpret_cast<const CUtensorMap*>(st.a_map),
-                                                            *reinterpret_cast<const CUtensorMap*>(st.w_map), P, H, V, m_tiles,
-                                                            n_tiles, keys);
-    e = cudaGetLastError();
-  }
+  if (e != cudaSuccess) return e;
+  const int m_tiles = (rows_extent + kBM - 1) / kBM, n_tiles = (V + kBN - 1) / kBN;
+  const int grid = m_tiles * n_tiles < num_sms ? m_tiles * n_tiles : num_sms;
+  lm_head_kernel<EPI><<<grid, kLmThreads, kLmSmem, s>>>(*reinterpret_cast<const CUtensorMap*>(st.a_map),
+                                                         *reinterpret_cast<const CUtensorMap*>(st.w_map), P, H, V, m_tiles, n_tiles, E);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int lm_head_vocab_tiles(int V) { return (V + kBN - 1) / kBN; }
+
+int launch_lm_head_argmax(const DevPlan& P, LmHeadState& st, const void* hidden, const void* weight, int H, int V, int rows_extent,
+                          int num_sms, unsigned long long* keys, float4* row_final, cudaStream_t s, std::string& err) {
+  if (rows_extent <= 0) return 0;
+  if (!refresh_maps(st, hidden, weight, H, V, rows_extent, err)) return 4;
+  LmEpilogue E{};
+  E.keys = keys;
+  E.rows = rows_extent;
+  cudaError_t e = cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)rows_extent, s);
+  if (e == cudaSuccess) e = launch_epilogue<kEpiArgmax>(st, P, H, V, rows_extent, num_sms, E, s);
   if (e == cudaSuccess) {
     lm_head_finish_kernel<<<(rows_extent + 255) / 256, 256, 0, s>>>(P, keys, row_final);
     e = cudaGetLastError();
   }
+  if (e != cudaSuccess) {
+    err = std::string("output projection launch: ") + cudaGetErrorString(e);
+    return 4;
+  }
+  return 0;
+}
+
+int launch_lm_head_stats(const DevPlan& P, LmHeadState& st, const void* hidden, const void* weight, int H, int V, int rows_extent,
+                         int num_sms, unsigned long long* keys, float2* tile_part, float* zd, const int32_t* draft_tokens,
+                         const float* temperature, float4* row_final, cudaStream_t s, std::string& err) {
+  if (rows_extent <= 0) return 0;
+  if (!refresh_maps(st, hidden, weight, H, V, rows_extent, err)) return 4;
+  LmEpilogue E{};
+  E.keys = keys;
+  E.tile_part = tile_part;
+  E.zd = zd;
+  E.draft_tokens = draft_tokens;
+  E.temperature = temperature;
+  E.rows = rows_extent;
+  cudaError_t e = cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)rows_extent, s);
+  if (e == cudaSuccess) e = launch_epilogue<kEpiStats>(st, P, H, V, rows_extent, num_sms, E, s);
+  if (e == cudaSuccess) {
+    lm_head_finish_stats_kernel<<<(rows_extent + 7) / 8, 256, 0, s>>>(P, keys, tile_part, lm_head_vocab_tiles(V), row_final);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    err = std::string("output projection launch: ") + cudaGetErrorString(e);
+    return 4;
+  }
+  return 0;
+}
+
+int launch_lm_head_recover_rows(const DevPlan& P, LmHeadState& st, const int32_t* recover_row, const void* hidden, void* hidden_rows,
+                                const void* weight, int H, int V, int batch_extent, int num_sms, float* logits, long long ld,
+                                cudaStream_t s, std::string& err) {
+  if (batch_extent <= 0) return 0;
+  if (!refresh_maps(st, hidden_rows, weight, H, V, batch_extent, err)) return 4;
+  lm_head_gather_rows_kernel<<<batch_extent, 128, 0, s>>>(P, recover_row, static_cast<const uint4*>(hidden),
+                                                          static_cast<uint4*>(hidden_rows), H / 8);
+  cudaError_t e = cudaGetLastError();
+  LmEpilogue E{};
+  E.store = logits;
+  E.store_ld = ld;
+  E.rows = batch_extent;
+  if (e == cudaSuccess) e = launch_epilogue<kEpiStore>(st, P, H, V, batch_extent, num_sms, E, s);
   if (e != cudaSuccess) {
     err = std::string("output projection launch: ") + cudaGetErrorString(e);
     return 4;
