@@ -272,13 +272,13 @@ __device__ __forceinline__ RecRow rec_row(const DevPlan& P, const AcceptArgs& A,
 // a common factor of the whole row and cancels in the normalisation): far inside what the fp64 sums and the comparison
 // against w * S can resolve.  An fp64 exponential (the library's, then a table and a degree-5 polynomial) and then fp64
 // arguments around ex2 kept these kernels bound by fp64 instructions.
-__device__ __forceinline__ double rec_exp_val(const RecRow& r, float x) {
-  return x == x ? (double)exp2f(fmaf(x, r.c, -r.mxc)) : 0.0;
-}
+__device__ __forceinline__ float rec_exp_f32(const RecRow& r, float x) { return x == x ? exp2f(fmaf(x, r.c, -r.mxc)) : 0.f; }
 // p_v and the recovery weight max(0, p_v - q_v) from the logit and the draft probability
 __device__ __forceinline__ void rec_weights_val(const RecRow& r, float x, double qv, double inv_den, double& p, double& res) {
-  p = rec_exp_val(r, x) * inv_den;
-  res = fmax(0.0, p - qv);
+  // (fp32 per entry, as in the cell sums this is compared with)
+  const float pf = rec_exp_f32(r, x) * (float)inv_den;
+  p = (double)pf;
+  res = (double)fmaxf(0.f, pf - (float)qv);
 }
 __device__ __forceinline__ void rec_weights(const RecRow& r, int v, double inv_den, double& p, double& res) {
   const double qv = r.q ? (double)r.q[v] : (v == r.onehot ? 1.0 : 0.0);
@@ -317,9 +317,10 @@ __global__ void __launch_bounds__(kRecThreads) recover_den_kernel(DevPlan P, Acc
 #pragma unroll
     for (int u = 0; u < 4; ++u)                         // four independent loads in flight per thread
       x[u] = load4(r.z, v0 + u * 4 * kRecThreads, end, vec, __int_as_float(0x7fc00000));
+    // (the terms carry the transcendental unit's 2^-22 anyway: four of them are added in fp32, the rest in fp64)
 #pragma unroll
     for (int u = 0; u < 4; ++u)
-      part += (rec_exp_val(r, x[u].x) + rec_exp_val(r, x[u].y)) + (rec_exp_val(r, x[u].z) + rec_exp_val(r, x[u].w));
+      part += (double)((rec_exp_f32(r, x[u].x) + rec_exp_f32(r, x[u].y)) + (rec_exp_f32(r, x[u].z) + rec_exp_f32(r, x[u].w)));
   }
   part = warp_sum_f64(part);
   __shared__ double sh[kRecThreads / 32];
@@ -341,7 +342,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, A
   const int a = A.recover_row[i];
   if (a < 0) return;
   const RecRow r = rec_row(P, A, i, a);
-  const double inv_den = 1.0 / rec_den(A, i);
+  const float inv_den32 = (float)(1.0 / rec_den(A, i));
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kWarps = kRecThreads / 32;
   const int V = A.vocab;
@@ -368,15 +369,17 @@ __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, A
       if (s < my_strips) {
         const int v = strip_at(s);
         // a one-hot draft distribution puts mass 1 on the drafted token
-        const double q0 = r.q ? (double)q[u].x : (v == r.onehot ? 1.0 : 0.0);
-        const double q1 = r.q ? (double)q[u].y : (v + 1 == r.onehot ? 1.0 : 0.0);
-        const double q2 = r.q ? (double)q[u].z : (v + 2 == r.onehot ? 1.0 : 0.0);
-        const double q3 = r.q ? (double)q[u].w : (v + 3 == r.onehot ? 1.0 : 0.0);
-        double p, res;
-        rec_weights_val(r, x[u].x, q0, inv_den, p, res); sp += p; sr += res;
-        rec_weights_val(r, x[u].y, q1, inv_den, p, res); sp += p; sr += res;
-        rec_weights_val(r, x[u].z, q2, inv_den, p, res); sp += p; sr += res;
-        rec_weights_val(r, x[u].w, q3, inv_den, p, res); sp += p; sr += res;
+        const float q0 = r.q ? q[u].x : (v == r.onehot ? 1.f : 0.f);
+        const float q1 = r.q ? q[u].y : (v + 1 == r.onehot ? 1.f : 0.f);
+        const float q2 = r.q ? q[u].z : (v + 2 == r.onehot ? 1.f : 0.f);
+        const float q3 = r.q ? q[u].w : (v + 3 == r.onehot ? 1.f : 0.f);
+        // Every term carries the transcendental unit's 2^-22 whatever follows, so p = e / den and max(0, p - q) are
+        // taken in fp32 and a lane's four entries added there; everything longer is summed in fp64.  (With all of it
+        // in fp64 this kernel was bound by fp64 instructions: seven per entry.)
+        const float p0 = rec_exp_f32(r, x[u].x) * inv_den32, p1 = rec_exp_f32(r, x[u].y) * inv_den32;
+        const float p2 = rec_exp_f32(r, x[u].z) * inv_den32, p3 = rec_exp_f32(r, x[u].w) * inv_den32;
+        sp += (double)((p0 + p1) + (p2 + p3));
+        sr += (double)((fmaxf(0.f, p0 - q0) + fmaxf(0.f, p1 - q1)) + (fmaxf(0.f, p2 - q2) + fmaxf(0.f, p3 - q3)));
         if ((s + 1) % strips_per_cell == 0) {            // the cell is complete
           const int cell = strip_cell(s);
           sp = warp_sum_f64(sp);

@@ -841,7 +841,7 @@ int as_accept_lm_head_sampled(as_plan_t* p, const void* hidden, const void* weig
   while ((vocab + chunk - 1) / chunk > p->accept_chunks_max) chunk *= 2;
   A.chunk_elems = chunk;
   A.chunks = (vocab + chunk - 1) / chunk;
-  int cell = 128;
+  int cell = 512;                            // (a cell costs its warp two fp64 reductions: few, large cells)
   while ((vocab + cell - 1) / cell > p->accept_cells_max) cell *= 2;
   A.cell_elems = cell;
   A.cells = (vocab + cell - 1) / cell;
@@ -904,7 +904,7 @@ int accept_impl(as_plan_t* p, const float* logits, int64_t ld, int vocab, const 
   A.recover_row = reinterpret_cast<int32_t*>(p->ws + p->off_recover);
   A.rec_den = reinterpret_cast<double*>(p->ws + p->off_rec_den);
   A.rec_cells = reinterpret_cast<double*>(p->ws + p->off_rec_cells);
-  int cell = 128;
+  int cell = 512;                            // (a cell costs its warp two fp64 reductions: few, large cells)
   while ((vocab + cell - 1) / cell > p->accept_cells_max) cell *= 2;
   A.cell_elems = cell;                       // a power of two below the chunk size, so it divides it
   A.cells = (vocab + cell - 1) / cell;
