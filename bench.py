@@ -32,11 +32,28 @@ from paper_2608_24004_b200 import workloads  # noqa: E402
 METRIC = "verified draft tokens/s per verify step"
 UNIT = "draft tokens/s"
 # DRAM bytes moved per algorithmic KV byte by the tensor-core attention kernels, from the ncu captures summarised in
-# profiles/: traffic grows in proportion to the KV bytes, so the ratio is scaled to the launch that is timed here.
-#   head_dim 128 (attn_tc_kernel), attn_tc_qwen3_8b_batch16_ncu_full.md: (721.08 MB read + 4.49 MB written) / 719.79 MB
-#   head_dim 64 (attn_rows_kernel), attn_rows_gpt_oss_20b_batch16_ncu_full.md: (1256.73 MB + 9.11 MB) / 1185.10 MB;
-#     the excess is the second walk over the keys of the requests with more than 128 query rows (1 in 17 there)
-ATTN_TC_DRAM_BYTES_PER_KV_BYTE = {128: 1.0094, 64: 1.0681}
+# profiles/ (batch-16 slices): traffic grows in proportion to the KV bytes, so the ratio is scaled to the launch timed here.
+#   head_dim 128 (attn_tc_kernel), attn_tc_qwen3_8b_batch16_ncu_full.md: (721.05 MB read + 4.21 MB written) / 719.79 MB
+#   head_dim 64 (attn_rows_kernel), attn_rows_gpt_oss_20b_batch16_ncu_full.md: 1.017 for requests of up to 128 query rows;
+#     a request with more is walked once per block of rows ((2375.1 + 15.7) / 1185.4 = 2.017 with every request at 136)
+ATTN_TC_DRAM_BYTES_PER_KV_BYTE = {128: 1.0076, 64: 1.017}
+
+
+def extra_walks_share(b, kind):
+    """Share of the layer's KV bytes that is read a second (third) time: requests whose query rows exceed what one launch
+    item holds are walked once per row block (head_dim 64: blocks of 128 rows; head_dim 128: blocks of at most 96 rows for
+    requests above 112 rows)."""
+    G = b.num_q_heads // b.num_kv_heads
+    rows = G * (b.draft_lens.astype(np.int64) + 1)
+    if b.head_dim == 64:
+        blocks = -(-rows // 128)
+    else:
+        blocks = np.where(rows > 112, -(-rows // 96), 1)
+    W = b.kinds[kind].window
+    vis = np.minimum(b.seq_lens.astype(np.int64) + b.draft_lens + 1, W + b.draft_lens if W > 0 else 1 << 60)
+    return float(((blocks - 1) * vis).sum() / max(vis.sum(), 1))
+
+
 HBM_NOMINAL_GBS = 8000.0
 
 
@@ -49,7 +66,7 @@ def measured_peaks():
 
 
 # hidden sizes of the models the workloads are shaped after
-HIDDEN_DIM = {"qwen3_8b": 4096, "r1_distill_llama_8b": 4096, "gpt_oss_20b": 2880, "tiny": 512}
+HIDDEN_DIM = {"qwen3_8b": 4096, "r1_distill_llama_8b": 4096, "gpt_oss_20b": 2880, "gpt_oss_20b_all_k16": 2880, "tiny": 512}
 
 
 def lm_head_leg(bnd, vs, b, workload, steps):
@@ -104,7 +121,7 @@ def roofline_of(bnd, b, vs, kind, attn_ms):
                 "algorithmic_bytes_per_launch": kv_bytes, "avg_launch_ms": attn_ms,
                 "ctas": stats["num_ctas"], "items": stats["num_items"], "merged_pairs": stats["num_merges"]}
     if roofline["kernel"] != "attn_simt":
-        roofline["traffic"] = ATTN_TC_DRAM_BYTES_PER_KV_BYTE[b.head_dim] * kv_bytes
+        roofline["traffic"] = (ATTN_TC_DRAM_BYTES_PER_KV_BYTE[b.head_dim] + extra_walks_share(b, kind)) * kv_bytes
         roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch on a batch-16 slice (ncu), "
                                     "divided by that launch's algorithmic KV bytes, times this batch's KV bytes")
     return roofline
@@ -225,6 +242,8 @@ def make_workload(name, device, seed_offset=0, batch=None, min_context=0):
         return workloads.r1_distill_llama_8b(device=device, seed=4000 + seed_offset, min_context=min_context, **over)
     if name == "gpt_oss_20b":
         return workloads.gpt_oss_20b(device=device, seed=3000 + seed_offset, **over)
+    if name == "gpt_oss_20b_all_k16":
+        return workloads.gpt_oss_20b(device=device, seed=3000 + seed_offset, all_max=True, **over)
     raise SystemExit(f"unknown workload {name}")
 
 

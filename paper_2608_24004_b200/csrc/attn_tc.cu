@@ -846,14 +846,20 @@ bool attn_tc_supported(int Hq, int Hkv, int D, int bs, int max_draft, int window
 int launch_attn_tc(const DevPlan& P, const AttnArgs& A, TcState& st, cudaStream_t s, std::string& err) {
   if (A.num_ctas == 0) return 0;
   AttnArgs B = A;
-  if (st.k_pool != A.k_pool || st.v_pool != A.v_pool) {
-    if (!encode_pool_map(st.k_map, A.k_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
-    if (!encode_pool_map(st.v_map, A.v_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
-    st.k_pool = A.k_pool;
-    st.v_pool = A.v_pool;
+  TcState::Entry* en = nullptr;
+  for (int x = 0; x < TcState::kEntries && !en; ++x)
+    if (st.entry[x].k_pool == A.k_pool && st.entry[x].v_pool == A.v_pool) en = &st.entry[x];
+  if (!en) {
+    en = &st.entry[st.next];
+    st.next = (st.next + 1) % TcState::kEntries;
+    en->k_pool = en->v_pool = nullptr;
+    if (!encode_pool_map(en->k_map, A.k_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
+    if (!encode_pool_map(en->v_map, A.v_pool, P.num_blocks, P.Hkv, P.bs, P.D, err)) return 4;
+    en->k_pool = A.k_pool;
+    en->v_pool = A.v_pool;
   }
-  const CUtensorMap& km = *reinterpret_cast<const CUtensorMap*>(st.k_map);
-  const CUtensorMap& vm = *reinterpret_cast<const CUtensorMap*>(st.v_map);
+  const CUtensorMap& km = *reinterpret_cast<const CUtensorMap*>(en->k_map);
+  const CUtensorMap& vm = *reinterpret_cast<const CUtensorMap*>(en->v_map);
   // the instance is as wide as this step's longest draft needs, not as the plan's maximum allows
   const int rows = A.rows_step > 0 ? A.rows_step : (P.Hq / P.Hkv) * (P.max_draft + 1);
   const cudaError_t e = attn_rows_on_m(P.D, rows) ? launch_rows_instance(km, vm, P, B, s) : launch_for_rows<128>(rows, km, vm, P, B, s);

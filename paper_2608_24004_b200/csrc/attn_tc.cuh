@@ -6,11 +6,18 @@
 
 namespace asv {
 
-struct TcState {             // per-plan cache: tensor maps are rebuilt only when a pool pointer changes
-  const void* k_pool = nullptr;
-  const void* v_pool = nullptr;
-  alignas(64) unsigned char k_map[128];
-  alignas(64) unsigned char v_map[128];
+// Per-plan cache of tensor maps, keyed by the pool pointers: a model's layers have a pool pair each and one plan
+// serves them in turn, so a single entry would be encoded anew (on the host, inside the step) at every call.
+struct TcState {
+  static constexpr int kEntries = 16;
+  struct Entry {
+    const void* k_pool = nullptr;
+    const void* v_pool = nullptr;
+    alignas(64) unsigned char k_map[128];
+    alignas(64) unsigned char v_map[128];
+  };
+  Entry entry[kEntries];
+  int next = 0;              // round-robin replacement
 };
 
 bool attn_tc_supported(int Hq, int Hkv, int D, int bs, int max_draft, int window);
