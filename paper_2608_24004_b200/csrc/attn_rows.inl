@@ -508,7 +508,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
     const int W = A.window;
     float2* const ml_all = reinterpret_cast<float2*>(smem + L::kOffMl);
     bool ok = true;
-    uint32_t g = 0;
+    uint32_t g_run = 0;                                   // running number of the current (item, row block)'s first tile
     // One arrival per warp, after every lane has done its part (each lane fences its own accesses first): 128 * NS
     // arrivals on one barrier word are 128 * NS serialised shared-memory atomics per tile.
     auto warp_arrive = [&](uint32_t bar) {
@@ -579,8 +579,11 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
         q_pending = true;
       }
 
-      for (int tile = 0; tile < v.tiles && ok; ++tile, ++g) {
-        if ((int)(g % NS) != stream) continue;            // the other stream's tile
+      // (only this stream's tiles are visited: a turn of this loop for the other stream's tile is a taken branch back over
+      // the whole softmax, which costs about 200 cycles of instruction fetch)
+      static_assert(NS == 2, "tile parity");
+      for (int tile = (int)((stream ^ g_run) & 1u); tile < v.tiles && ok; tile += NS) {
+        const uint32_t g = g_run + tile;
         const int kbase = v.key_begin + tile * kTile;
         const int sbuf = g & 1, pbuf = g % NP;
         if (!mbar_wait_c(bar_s_full(sbuf), (g >> 1) & 1u, ctl, P.status, 9)) { ok = false; break; }
@@ -838,6 +841,7 @@ attn_rows_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant
         }
       }
       if (!ok) break;
+      g_run += v.tiles;
       if (q_pending) load_q_finish(item_idx + 1);         // (a block in which this stream had no tile)
 
       // ---- epilogue: merge the streams' (m, l, O_s) of every row; thread (stream, r) finishes D / NS columns of row r ----
