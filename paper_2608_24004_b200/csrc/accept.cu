@@ -253,6 +253,7 @@ struct RecRow {
   int onehot;            // ... or the drafted token when the draft distribution is one-hot, else -1
   float c, mxc;          // log2(e) / T and the row maximum of z times it: 2^(z c - mxc) = exp(z / T - max)
   bool bonus;            // all drafts accepted: draw from p itself
+  double den;            // softmax denominator of the row against mxc
 };
 __device__ __forceinline__ RecRow rec_row(const DevPlan& P, const AcceptArgs& A, int i, int a) {
   const ReqMeta rq = P.req[i];
@@ -265,7 +266,11 @@ __device__ __forceinline__ RecRow rec_row(const DevPlan& P, const AcceptArgs& A,
   // the largest logit of the row is known from the first pass (NaN never wins there either)
   const double c = 1.4426950408889634 / (double)A.temperature[i];
   r.c = (float)c;
-  r.mxc = (float)((double)A.row_final[row].x * c);
+  const float4 rf = A.row_final[row];
+  r.mxc = (float)((double)rf.x * c);
+  // The denominator is the first pass's: the online (reference, sum of 2^(z c - reference)) of the row, moved to this
+  // reference (the two references differ by a rounding at most).  An fp32 sum, like the ratio the drafts were judged by.
+  r.den = (double)rf.w * (double)exp2f(rf.z - r.mxc);
   return r;
 }
 // exp(z_v / T - max); 0 for NaN.  One fp32 FMA and the transcendental unit (about 2^-22 relative; the rounding of mxc is
@@ -296,44 +301,7 @@ __device__ __forceinline__ float4 load4(const float* row, int v, int V, bool vec
   return o;
 }
 __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
-__device__ __forceinline__ double rec_den(const AcceptArgs& A, int i) {     // chunk sums in chunk order
-  double den = 0.0;
-  for (int c = 0; c < A.chunks; ++c) den += A.rec_den[(size_t)i * A.chunks + c];
-  return den;
-}
-
-// Recovery, step 1: softmax denominator of row a_i in fp64, one CTA per vocabulary chunk.
-__global__ void __launch_bounds__(kRecThreads) recover_den_kernel(DevPlan P, AcceptArgs A) {
-  const int i = blockIdx.x / A.chunks, chunk = blockIdx.x - i * A.chunks;
-  if (i >= P.hdr->batch) return;
-  const int a = A.recover_row[i];
-  if (a < 0) return;
-  const RecRow r = rec_row(P, A, i, a);
-  const int begin = chunk * A.chunk_elems, end = min(begin + A.chunk_elems, A.vocab);
-  const bool vec = aligned16(r.z);
-  double part = 0.0;
-  for (int v0 = begin + threadIdx.x * 4; v0 < end; v0 += 16 * kRecThreads) {
-    float4 x[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u)                         // four independent loads in flight per thread
-      x[u] = load4(r.z, v0 + u * 4 * kRecThreads, end, vec, __int_as_float(0x7fc00000));
-    // (the terms carry the transcendental unit's 2^-22 anyway: four of them are added in fp32, the rest in fp64)
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      part += (double)((rec_exp_f32(r, x[u].x) + rec_exp_f32(r, x[u].y)) + (rec_exp_f32(r, x[u].z) + rec_exp_f32(r, x[u].w)));
-  }
-  part = warp_sum_f64(part);
-  __shared__ double sh[kRecThreads / 32];
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = part;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double tot = 0.0;
-    for (int wv = 0; wv < kRecThreads / 32; ++wv) tot += sh[wv];
-    A.rec_den[(size_t)i * A.chunks + chunk] = tot;
-  }
-}
-
-// Recovery, step 2: per cell (cell_elems consecutive vocabulary entries, a multiple of 128) the mass of p and
+// Recovery, step 1: per cell (cell_elems consecutive vocabulary entries, a multiple of 128) the mass of p and
 // of max(0, p - q).  A warp owns whole cells and walks them in strips of 128 entries, four entries per lane,
 // four strips' loads in flight; the sums do not depend on the launch shape.
 __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, AcceptArgs A) {
@@ -342,7 +310,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, A
   const int a = A.recover_row[i];
   if (a < 0) return;
   const RecRow r = rec_row(P, A, i, a);
-  const float inv_den32 = (float)(1.0 / rec_den(A, i));
+  const float inv_den32 = (float)(1.0 / r.den);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kWarps = kRecThreads / 32;
   const int V = A.vocab;
@@ -397,7 +365,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_cells_kernel(DevPlan P, A
   }
 }
 
-// Recovery, step 3: one warp per request walks the cell sums to the cell that holds w * S and scans it.
+// Recovery, step 2: one warp per request walks the cell sums to the cell that holds w * S and scans it.
 __global__ void recover_pick_kernel(DevPlan P, AcceptArgs A) {
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -405,7 +373,7 @@ __global__ void recover_pick_kernel(DevPlan P, AcceptArgs A) {
   const int a = A.recover_row[i];
   if (a < 0) return;
   const RecRow r = rec_row(P, A, i, a);
-  const double inv_den = 1.0 / rec_den(A, i);
+  const double inv_den = 1.0 / r.den;
   const double* cells = A.rec_cells + (size_t)i * A.cells * 2;
   const int ncell = (A.vocab + A.cell_elems - 1) / A.cell_elems;
   const int per = (ncell + 31) / 32;
@@ -491,9 +459,6 @@ cudaError_t launch_accept(const DevPlan& P, const AcceptArgs& A, cudaStream_t s)
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (A.temperature) {
-    recover_den_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     recover_cells_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -505,11 +470,8 @@ cudaError_t launch_accept(const DevPlan& P, const AcceptArgs& A, cudaStream_t s)
 
 cudaError_t launch_recover(const DevPlan& P, const AcceptArgs& A, cudaStream_t s) {
   if (P.batch == 0) return cudaSuccess;
-  recover_den_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
   recover_cells_kernel<<<(unsigned)A.chunks * (unsigned)P.batch, kRecThreads, 0, s>>>(P, A);
-  e = cudaGetLastError();
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   recover_pick_kernel<<<(P.batch + 3) / 4, 128, 0, s>>>(P, A);
   return cudaGetLastError();

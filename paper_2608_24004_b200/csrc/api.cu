@@ -84,7 +84,7 @@ struct as_plan_s {
   char* ws = nullptr;
   size_t ws_bytes = 0;
   size_t off_status = 0, off_meta = 0, meta_capacity = 0, off_commit_counts = 0, off_part_o = 0, off_part_ml = 0,
-         off_row_part = 0, off_row_final = 0, off_row_ticket = 0, off_recover = 0, off_rec_den = 0, off_rec_cells = 0, total_bytes = 0;
+         off_row_part = 0, off_row_final = 0, off_row_ticket = 0, off_recover = 0, off_rec_cells = 0, total_bytes = 0;
   // current step
   bool planned = false;
   int batch = 0, total_q = 0, total_d = 0;
@@ -342,8 +342,6 @@ int as_plan_create(as_plan_t** out, const as_layer_desc* kinds, int num_kinds, i
   off += align_up(sizeof(int32_t) * (size_t)p->max_total_q, 256);
   p->off_recover = off;
   off += align_up(sizeof(int32_t) * max_batch, 256);
-  p->off_rec_den = off;
-  off += align_up(sizeof(double) * (size_t)max_batch * p->accept_chunks_max, 256);
   p->off_rec_cells = off;
   off += align_up(sizeof(double) * 2 * (size_t)max_batch * p->accept_cells_max, 256);
   p->total_bytes = off;
@@ -832,7 +830,6 @@ int as_accept_lm_head_sampled(as_plan_t* p, const void* hidden, const void* weig
   A.out_tokens = out_tokens;
   A.row_final = reinterpret_cast<float4*>(p->ws + p->off_row_final);
   A.recover_row = reinterpret_cast<int32_t*>(p->ws + p->off_recover);
-  A.rec_den = reinterpret_cast<double*>(p->ws + p->off_rec_den);
   A.rec_cells = reinterpret_cast<double*>(p->ws + p->off_rec_cells);
   A.zd = zd;
   A.rec_logits = rec_logits;
@@ -857,7 +854,7 @@ int as_accept_lm_head_sampled(as_plan_t* p, const void* hidden, const void* weig
                                    rec_logits, (long long)rec_ld, s, err);
   if (rc != 0) return fail(rc, "as_accept_lm_head_sampled: " + err);
   AS_CUDA(launch_recover(d, A, s));
-  p->launches += 9;
+  p->launches += 8;
   return AS_OK;
 }
 
@@ -902,14 +899,13 @@ int accept_impl(as_plan_t* p, const float* logits, int64_t ld, int vocab, const 
   A.chunk_elems = chunk;
   A.chunks = (vocab + chunk - 1) / chunk;
   A.recover_row = reinterpret_cast<int32_t*>(p->ws + p->off_recover);
-  A.rec_den = reinterpret_cast<double*>(p->ws + p->off_rec_den);
   A.rec_cells = reinterpret_cast<double*>(p->ws + p->off_rec_cells);
   int cell = 512;                            // (a cell costs its warp two fp64 reductions: few, large cells)
   while ((vocab + cell - 1) / cell > p->accept_cells_max) cell *= 2;
   A.cell_elems = cell;                       // a power of two below the chunk size, so it divides it
   A.cells = (vocab + cell - 1) / cell;
   AS_CUDA(launch_accept(dev_plan(p), A, static_cast<cudaStream_t>(stream)));
-  p->launches += temperature ? 5 : 2;
+  p->launches += temperature ? 4 : 2;
   return AS_OK;
 }
 }  // namespace

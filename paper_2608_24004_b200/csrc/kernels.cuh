@@ -56,7 +56,6 @@ struct AcceptArgs {
   int32_t* row_ticket;        // [total_q] chunks finished so far; zero between calls
   int32_t chunks, chunk_elems;
   int32_t* recover_row;       // [batch] row whose recovery distribution must be sampled, or -1
-  double* rec_den;            // [batch, chunks] fp64 softmax denominator of that row, per chunk
   double* rec_cells;          // [batch, cells, 2] mass of p and of max(0, p - q) per cell of cell_elems entries
   int32_t cells, cell_elems;  // cell_elems divides chunk_elems
 };
