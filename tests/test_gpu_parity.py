@@ -108,6 +108,7 @@ SHAPES = [
     (64, 8, 128, 16, 0, False, [700, 2600, 127], [23, 17, 31]),      # 192, 144 and 256 rows at head_dim 128
     (64, 8, 128, 32, 200, True, [40000, 199, 200, 201], [31, 16, 24, 5]),   # row blocks under a window, one long split pair
     (48, 16, 128, 16, 0, False, [900, 300], [60, 41]),               # three query heads per kv head: blocks of 42 positions
+    (16, 2, 64, 128, 0, False, [260, 4000, 130], [2, 9, 0]),         # head_dim 64 with one page per tile
 ]
 
 
