@@ -19,11 +19,14 @@
 // row, its own S and P buffer and its OWN accumulator O_s in TMEM.  The streams never talk to each other during an
 // item; the epilogue merges the (m, l, O_s) triples of a row like split-KV partials.
 //
-// Softmax of a tile, per thread: pass 1 takes the row maximum of the 128 scores; the row's reference follows it
-// lazily (it moves, and O_s and the row sum are rescaled, only when the maximum exceeds it by more than 2^8); pass 2
-// turns the scores into weights 2^(score - reference).  The scores have left tensor memory for good a quarter of
-// the way before the end of pass 2; from then on the stream's S buffer is free (s_free) and the QK product of the
-// stream's next tile runs under the rest of this tile's weights.
+// Softmax of a tile, per thread: the weights 2^(score - reference) are computed against the row's reference as it
+// stands, with no pass for the maximum.  A row whose weights of the tile add up to more than 2^9 keeps them (bf16 keeps
+// their relative precision, O_s and the sum are fp32) and moves its reference afterwards: the sum at once, its row of
+// O_s when the tile's PV product has completed.  Weights that may have overflowed (a score 2^96 above its reference)
+// are recomputed from the queries and keys in global memory.  Only a stream's first tile of an item, a row that has
+// seen no key yet and the masked edge tiles take the row maximum first.  The scores have left tensor memory for good
+// a quarter of the way before the weights are finished; from then on the stream's S buffer is free (s_free) and the
+// QK product of the stream's next tile runs under the rest of this tile's weights.
 //
 // K and V tiles travel in separate rings (3 + 8 slots of 16 KB), each filled by its own producer warp: a K tile is
 // dead as soon as its QK product has completed, a V tile has to wait for the whole softmax of its tile, and in one
@@ -31,9 +34,10 @@
 // not the arithmetic, bounded the kernel then (five fused slots: 1590 cycles a tile, four: 1820).
 //
 // Warps (352 threads, one CTA per SM, persistent): 0..7 softmax (stream = warp / 4, TMEM lane quarter = warp % 4),
-// 8 K producer, 9 V producer, 10 issues every tcgen05.mma from one lane.  Issuing a product costs that lane 50 cycles
-// when it has its scheduler to itself and up to twice that when softmax warps compete for the issue slots; at twelve
-// products a tile it is what bounds wide tiles.  A warp's scheduler is its index modulo 4, and so is its TMEM lane
+// 8 K producer, 9 V producer, 10 issues every tcgen05.mma from one lane.  That lane's own instructions are what bounds
+// the kernel (measured: cycles added to it show one to one in the time of a tile, the softmax arithmetic taken out
+// shows nothing): a product costs it 50 cycles when it has its scheduler to itself and more when softmax warps compete
+// for the issue slots, a commit about a hundred, a turn of its loop a few hundred.  A warp's scheduler is its index modulo 4, and so is its TMEM lane
 // quarter: warp 10 shares scheduler 2 with the softmax warps of lanes 64..95, and the block's rows 96..127, the ones
 // that most items do not have, are mapped to those lanes (rows 64..95 to lanes 96..127).
 // Every wait is bounded as in the other kernel.
