@@ -10,10 +10,11 @@
 //   rejection, and greedy requests get their extra token.  Sampling requests record which row must be
 //   re-read.
 // Stage 3 (recover): a sampling request draws its extra token from max(0, p - q) (or p) by inverse CDF.
-//   That row alone is re-read, with fp64 softmax and fp64 accumulation, so that the chosen index does not
-//   depend on how a long fp32 prefix sum would have rounded.  Three small launches, all spread over the
-//   vocabulary chunks so that every SM takes part: the denominator, the mass of each cell of consecutive
-//   entries, then one warp per request walks the cell sums to the cell holding w * S and scans only that.
+//   That row alone is re-read.  Entries are weighed in fp32 (four at a time) and summed in fp64 in index order, so that
+//   the chosen index does not depend on how a long fp32 prefix sum would have rounded; the softmax denominator is
+//   stage 1's.  Two small launches: the mass of each cell of consecutive entries, spread over the vocabulary chunks
+//   so that every SM takes part, then one warp per request walks the cell sums to the cell holding w * S and scans
+//   only that.
 #include "kernels.cuh"
 #include "lm_head.cuh"
 
